@@ -1,0 +1,173 @@
+/*
+ * dst -- densify assumed-sparse (IndexedSlices) gradients on one NVIDIA B200.
+ *
+ * The operation is the one the paper "Densifying Assumed-sparse Tensors"
+ * (arXiv 1905.04035) introduces in Section 4 / Listing 1: a gradient held as
+ * IndexedSlices (row indices + [n_rows, d] value rows, Section 3) is converted
+ * to a dense [vocab, d] tensor so that gradients are accumulated by reduction
+ * (Algorithm 1, "reduce" branch) instead of by concatenation ("gather" branch).
+ * For the tied embedding / pre-softmax projection weight of Section 3 the
+ * dense partner is the projection gradient, added in the same pass:
+ *
+ *     out[v, c] = (dense_in ? dense_in[v, c] : 0)
+ *               + sum over slices r and rows i with indices_r[i] == v of values_r[i, c]
+ *
+ * Conventions for every entry point
+ *   - All tensor arguments are DEVICE pointers unless a comment says "host".
+ *     Buffers are owned by the caller; the library never allocates, frees or
+ *     synchronises.  All work is enqueued on `stream`.
+ *   - values_r is row-major contiguous [n_rows_r, d]; dense_in and out are
+ *     row-major contiguous [vocab, d] in `out_type`; inputs are read-only.
+ *   - `out` may alias `dense_in` (in-place accumulate).  It must not overlap
+ *     indices, values or the workspace.
+ *   - Duplicate indices are summed.  Rows whose index lies outside [0, vocab)
+ *     are skipped and counted (result->n_out_of_range, result->status =
+ *     DST_ERR_INDEX_OUT_OF_RANGE); they never fault.
+ *   - The summation order is fixed by the shapes alone (ascending input
+ *     position inside fixed-size chunks, a fixed combine tree, dense_in last),
+ *     so two calls on the same inputs give bit-identical results, and
+ *     dst_densify_concat equals dst_densify on the physical concatenation.
+ *   - Return value: DST_OK when everything was enqueued.  Problems found on
+ *     the host (bad argument, workspace too small, unsupported type) return an
+ *     error and enqueue nothing.  Problems found on the device are reported in
+ *     `result` once the stream has run.
+ *   - The fast kernels need 16-byte aligned base pointers and row sizes that
+ *     are multiples of 16 bytes; other shapes take a slow scalar kernel.
+ */
+#ifndef DST_H_
+#define DST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DST_OK = 0,
+    DST_ERR_INVALID_ARG = 1,
+    DST_ERR_UNSUPPORTED = 2,
+    DST_ERR_WORKSPACE_TOO_SMALL = 3,
+    DST_ERR_INDEX_OUT_OF_RANGE = 4, /* device-side: some rows were skipped */
+    DST_ERR_TIMEOUT = 5,            /* device-side: a bounded wait gave up; output invalid */
+    DST_ERR_CUDA = 6
+} dst_status_t;
+
+typedef enum { DST_I32 = 0, DST_I64 = 1 } dst_index_t;
+typedef enum { DST_F32 = 0, DST_BF16 = 1 } dst_dtype_t;
+
+/* Element types.  Accumulation is always fp32.  flags must be 0. */
+typedef struct {
+    int32_t index_type; /* dst_index_t: type of indices and of unique_rows */
+    int32_t value_type; /* dst_dtype_t: type of the value rows */
+    int32_t out_type;   /* dst_dtype_t: type of dense_in and out */
+    uint32_t flags;
+} dst_opts_t;
+
+/* One IndexedSlices object (Section 3): device pointers. */
+typedef struct {
+    const void* indices; /* [n_rows] */
+    const void* values;  /* [n_rows, d] */
+    int64_t n_rows;
+} dst_slice_t;
+
+/* Written by the device when the enqueued work runs (device or pinned host memory). */
+typedef struct {
+    int32_t status;         /* dst_status_t */
+    int32_t n_unique;       /* number of distinct valid rows */
+    int64_t n_out_of_range; /* input rows skipped */
+    int64_t max_segment;    /* largest number of input rows naming one output row */
+} dst_result_t;
+
+/* Footprints in bytes (Section 4, Fig. 5a: gather of slices vs one dense tensor). */
+typedef struct {
+    int64_t n_rows_total;
+    int64_t sparse_value_bytes;     /* sum_r n_rows_r * d * sizeof(value) */
+    int64_t sparse_index_bytes;     /* sum_r n_rows_r * sizeof(index) */
+    int64_t sparse_bytes;           /* the two above */
+    int64_t dense_bytes;            /* vocab * d * sizeof(out) */
+    int64_t gather_all_value_bytes; /* sum_r (vocab + n_rows_r) * d * sizeof(value): Algorithm 1's
+                                       gather branch also turns the dense partner into vocab slices */
+    double sparse_over_dense;
+    double gather_all_over_dense;
+} dst_bytes_report_t;
+
+typedef struct CUstream_st* dst_stream_t; /* a cudaStream_t */
+
+int dst_version(void);
+const char* dst_status_string(int status);
+
+/* Bytes of device workspace dst_densify / dst_densify_concat need for inputs of
+ * at most n_rows_total rows in R slices.  Returns 0 for invalid arguments. */
+size_t dst_workspace_bytes(int64_t n_rows_total, int32_t R, int64_t d, int64_t vocab, const dst_opts_t* opts);
+
+/*
+ * Densify one IndexedSlices gradient and add the dense partner
+ * (Section 4, Listing 1: convert_to_tensor of an IndexedSlices; Algorithm 1 line 4: sum).
+ *   indices [n_rows], values [n_rows, d], dense_in [vocab, d] or NULL, out [vocab, d].
+ *   workspace: >= dst_workspace_bytes(n_rows, 1, d, vocab, opts) bytes, 256-byte aligned.
+ *   unique_rows (index_type) / counts (int32): optional outputs with room for
+ *   min(n_rows, vocab) entries -- the distinct valid rows in ascending order and
+ *   how many input rows named each.  result: optional.
+ * n_rows == 0 gives out = dense_in (or zeros).  vocab == 0 or d == 0 is a no-op.
+ */
+int dst_densify(const void* indices, const void* values, int64_t n_rows, int64_t d, int64_t vocab,
+                const void* dense_in, void* out, dst_stream_t stream, const dst_opts_t* opts,
+                void* workspace, size_t workspace_bytes,
+                void* unique_rows, int32_t* counts, dst_result_t* result);
+
+/*
+ * Same, for the R slices a sparse gather would have concatenated (Algorithm 1
+ * line 6; the cross-rank gather of Section 3).  `slices` is a HOST array of R
+ * descriptors holding device pointers; it is read during the call only.  No
+ * concatenated copy is made; the result is bit-identical to dst_densify on the
+ * physical concatenation in slice order.  Empty slices are allowed.  R == 0
+ * behaves like n_rows == 0.
+ */
+int dst_densify_concat(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab,
+                       const void* dense_in, void* out, dst_stream_t stream, const dst_opts_t* opts,
+                       void* workspace, size_t workspace_bytes,
+                       void* unique_rows, int32_t* counts, dst_result_t* result);
+
+/* Bytes of device staging memory dst_densify_concat_host needs. */
+size_t dst_host_staging_bytes(int64_t n_rows_total, int64_t d, int64_t vocab, const dst_opts_t* opts);
+
+/*
+ * End-to-end variant for callers whose gradients live in HOST memory: `slices`
+ * holds HOST pointers, host_dense_in (nullable) and host_out are HOST buffers
+ * (pinned memory makes the copies asynchronous).  Enqueues host-to-device
+ * copies of every slice and of dense_in into `staging`, the densify itself,
+ * and the device-to-host copy of the result; host_result (nullable, host)
+ * receives the dst_result_t.  Nothing is synchronised: host_out is valid once
+ * `stream` has drained.  staging: >= dst_host_staging_bytes(...) device bytes.
+ */
+int dst_densify_concat_host(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab,
+                            const void* host_dense_in, void* host_out, dst_stream_t stream,
+                            const dst_opts_t* opts, void* staging, size_t staging_bytes,
+                            void* workspace, size_t workspace_bytes, dst_result_t* host_result);
+
+/*
+ * Footprint report (Section 4: 11.4 GB gathered vs 139 MB dense at 64 processes).
+ * n_rows_per_slice: HOST array of R row counts.  report: HOST.  Pure host arithmetic.
+ */
+int dst_bytes_report(const int64_t* n_rows_per_slice, int32_t R, int64_t d, int64_t vocab,
+                     const dst_opts_t* opts, dst_bytes_report_t* report);
+
+/*
+ * Measurement hooks (the paper instruments its runs with Horovod timelines, Section 3
+ * Fig. 3; these are the equivalent for this library).
+ *
+ * dst_profile_events: give two cudaEvent_t handles; every later densify call made by
+ * this host thread records `before` right before and `after` right after the
+ * row-reduction kernel (the kernel that moves the value, dense_in and out rows) on
+ * the call's stream.  Pass NULL, NULL to switch it off (the default).
+ * dst_kernel_launches: number of kernels this library has launched in this process.
+ */
+void dst_profile_events(void* before, void* after);
+int64_t dst_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DST_H_ */

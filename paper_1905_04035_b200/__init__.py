@@ -1,0 +1,25 @@
+"""B200-native densification of assumed-sparse (IndexedSlices) gradients.
+
+Thin binding over the C-ABI library declared in ``include/dst.h``: the Python
+functions carry the same names as the C entry points and only marshal
+arguments.  PyTorch supplies device memory and streams; every step of the
+operation runs in the library's CUDA kernels.  There is no CPU fallback: if
+the library has not been built, calls raise.
+"""
+from .binding import (  # noqa: F401
+    DST_STATUS,
+    Densifier,
+    DstError,
+    dst_bytes_report,
+    dst_densify,
+    dst_densify_concat,
+    dst_densify_concat_host,
+    dst_host_staging_bytes,
+    dst_kernel_launches,
+    dst_profile_events,
+    dst_status_string,
+    dst_version,
+    dst_workspace_bytes,
+    library_path,
+    load_library,
+)

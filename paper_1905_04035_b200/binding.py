@@ -1,0 +1,295 @@
+"""ctypes marshalling for ``libdst_b200.so`` (see ``include/dst.h`` for the contract)."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libdst_b200.so")
+_lib = None
+
+DST_STATUS = {
+    0: "DST_OK", 1: "DST_ERR_INVALID_ARG", 2: "DST_ERR_UNSUPPORTED", 3: "DST_ERR_WORKSPACE_TOO_SMALL",
+    4: "DST_ERR_INDEX_OUT_OF_RANGE", 5: "DST_ERR_TIMEOUT", 6: "DST_ERR_CUDA",
+}
+DST_I32, DST_I64 = 0, 1
+DST_F32, DST_BF16 = 0, 1
+
+
+class DstError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (%s)" % (where, DST_STATUS.get(status, status), dst_status_string(status)))
+
+
+class _Opts(ctypes.Structure):
+    _fields_ = [("index_type", ctypes.c_int32), ("value_type", ctypes.c_int32), ("out_type", ctypes.c_int32),
+                ("flags", ctypes.c_uint32)]
+
+
+class _Slice(ctypes.Structure):
+    _fields_ = [("indices", ctypes.c_void_p), ("values", ctypes.c_void_p), ("n_rows", ctypes.c_int64)]
+
+
+class _Result(ctypes.Structure):
+    _fields_ = [("status", ctypes.c_int32), ("n_unique", ctypes.c_int32), ("n_out_of_range", ctypes.c_int64),
+                ("max_segment", ctypes.c_int64)]
+
+
+class _BytesReport(ctypes.Structure):
+    _fields_ = [("n_rows_total", ctypes.c_int64), ("sparse_value_bytes", ctypes.c_int64),
+                ("sparse_index_bytes", ctypes.c_int64), ("sparse_bytes", ctypes.c_int64),
+                ("dense_bytes", ctypes.c_int64), ("gather_all_value_bytes", ctypes.c_int64),
+                ("sparse_over_dense", ctypes.c_double), ("gather_all_over_dense", ctypes.c_double)]
+
+
+RESULT_BYTES = ctypes.sizeof(_Result)
+
+# name -> (restype, argtypes); also the list of symbols the header declares
+_vp, _i64, _i32, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
+SYMBOLS = {
+    "dst_version": (ctypes.c_int, []),
+    "dst_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "dst_workspace_bytes": (_sz, [_i64, _i32, _i64, _i64, ctypes.POINTER(_Opts)]),
+    "dst_densify": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i64, _vp, _vp, _vp, ctypes.POINTER(_Opts), _vp, _sz,
+                                   _vp, _vp, _vp]),
+    "dst_densify_concat": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, _vp,
+                                          ctypes.POINTER(_Opts), _vp, _sz, _vp, _vp, _vp]),
+    "dst_host_staging_bytes": (_sz, [_i64, _i64, _i64, ctypes.POINTER(_Opts)]),
+    "dst_densify_concat_host": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, _vp,
+                                               ctypes.POINTER(_Opts), _vp, _sz, _vp, _sz, _vp]),
+    "dst_profile_events": (None, [_vp, _vp]),
+    "dst_kernel_launches": (ctypes.c_int64, []),
+    "dst_bytes_report": (ctypes.c_int, [ctypes.POINTER(_i64), _i32, _i64, _i64, ctypes.POINTER(_Opts),
+                                        ctypes.POINTER(_BytesReport)]),
+}
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load the CUDA library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(
+                "%s is missing: build it with `python -m paper_1905_04035_b200.build` "
+                "(nvcc, sm_100a). There is no CPU fallback." % _LIB_PATH)
+        lib = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _index_type(t: torch.dtype) -> int:
+    if t == torch.int64:
+        return DST_I64
+    if t == torch.int32:
+        return DST_I32
+    raise TypeError("indices must be int32 or int64, got %s" % t)
+
+
+def _dtype(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return DST_F32
+    if t == torch.bfloat16:
+        return DST_BF16
+    raise TypeError("values / dense tensors must be float32 or bfloat16, got %s" % t)
+
+
+def _opts(index_dtype, value_dtype, out_dtype) -> _Opts:
+    return _Opts(_index_type(index_dtype), _dtype(value_dtype), _dtype(out_dtype), 0)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_handle(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def dst_version() -> int:
+    return int(load_library().dst_version())
+
+
+def dst_status_string(status: int) -> str:
+    return load_library().dst_status_string(int(status)).decode()
+
+
+def dst_profile_events(before=None, after=None) -> None:
+    """Record two ``torch.cuda.Event`` objects around the row-reduction kernel of later calls
+    made from this thread; ``None, None`` switches it off.  The events must have been recorded
+    once already (torch creates the CUDA event lazily)."""
+    def handle(ev):
+        return None if ev is None else ctypes.c_void_p(ev.cuda_event)
+    load_library().dst_profile_events(handle(before), handle(after))
+
+
+def dst_kernel_launches() -> int:
+    return int(load_library().dst_kernel_launches())
+
+
+def dst_workspace_bytes(n_rows_total: int, R: int, d: int, vocab: int, index_dtype=torch.int64,
+                        value_dtype=torch.float32, out_dtype=torch.float32) -> int:
+    o = _opts(index_dtype, value_dtype, out_dtype)
+    return int(load_library().dst_workspace_bytes(n_rows_total, R, d, vocab, ctypes.byref(o)))
+
+
+def dst_host_staging_bytes(n_rows_total: int, d: int, vocab: int, index_dtype=torch.int64,
+                           value_dtype=torch.float32, out_dtype=torch.float32) -> int:
+    o = _opts(index_dtype, value_dtype, out_dtype)
+    return int(load_library().dst_host_staging_bytes(n_rows_total, d, vocab, ctypes.byref(o)))
+
+
+def dst_bytes_report(n_rows_per_slice: Sequence[int], d: int, vocab: int, index_dtype=torch.int64,
+                     value_dtype=torch.float32, out_dtype=torch.float32) -> dict:
+    o = _opts(index_dtype, value_dtype, out_dtype)
+    R = len(n_rows_per_slice)
+    arr = (ctypes.c_int64 * max(R, 1))(*[int(n) for n in n_rows_per_slice])
+    rep = _BytesReport()
+    rc = load_library().dst_bytes_report(arr, R, d, vocab, ctypes.byref(o), ctypes.byref(rep))
+    if rc != 0:
+        raise DstError(rc, "dst_bytes_report")
+    out = {name: getattr(rep, name) for name, _ in _BytesReport._fields_}
+    out["R"] = R
+    return out
+
+
+def _check_slice(idx: torch.Tensor, val: torch.Tensor, d: int, device) -> None:
+    if idx.dim() != 1 or not idx.is_contiguous() or not val.is_contiguous():
+        raise ValueError("indices must be 1-D contiguous and values contiguous")
+    if val.numel() != idx.shape[0] * d:
+        raise ValueError("values must be [n_rows, d]")
+    if idx.device != device or val.device != device:
+        raise ValueError("all tensors must live on the same device")
+
+
+def dst_densify_concat(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]], d: int, vocab: int,
+                       dense_in: Optional[torch.Tensor], out: torch.Tensor, workspace: torch.Tensor,
+                       unique_rows: Optional[torch.Tensor] = None, counts: Optional[torch.Tensor] = None,
+                       result: Optional[torch.Tensor] = None, stream=None,
+                       index_dtype: Optional[torch.dtype] = None, value_dtype: Optional[torch.dtype] = None) -> None:
+    """Enqueue ``dst_densify_concat`` (include/dst.h).  All tensors are CUDA tensors owned by the caller.
+
+    ``result``: an int32/uint8 CUDA (or pinned) tensor of at least 24 bytes that receives ``dst_result_t``.
+    """
+    lib = load_library()
+    R = len(slices)
+    if R:
+        index_dtype, value_dtype = slices[0][0].dtype, slices[0][1].dtype
+    elif index_dtype is None or value_dtype is None:
+        index_dtype, value_dtype = index_dtype or torch.int64, value_dtype or out.dtype
+    arr = (_Slice * max(R, 1))()
+    for r, (idx, val) in enumerate(slices):
+        if idx.dtype != index_dtype or val.dtype != value_dtype:
+            raise TypeError("all slices must share index and value dtypes")
+        _check_slice(idx, val, d, out.device)
+        arr[r].indices, arr[r].values, arr[r].n_rows = idx.data_ptr(), val.data_ptr(), idx.shape[0]
+    if out.numel() != vocab * d or not out.is_contiguous():
+        raise ValueError("out must be contiguous [vocab, d]")
+    if dense_in is not None and (dense_in.dtype != out.dtype or dense_in.numel() != vocab * d
+                                 or not dense_in.is_contiguous()):
+        raise ValueError("dense_in must be contiguous [vocab, d] in out's dtype")
+    o = _opts(index_dtype, value_dtype, out.dtype)
+    with torch.cuda.device(out.device):
+        rc = lib.dst_densify_concat(arr, R, d, vocab, _ptr(dense_in), _ptr(out), _stream_handle(stream),
+                                    ctypes.byref(o), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                    _ptr(unique_rows), _ptr(counts), _ptr(result))
+    if rc != 0:
+        raise DstError(rc, "dst_densify_concat")
+
+
+def dst_densify(indices: torch.Tensor, values: torch.Tensor, d: int, vocab: int,
+                dense_in: Optional[torch.Tensor], out: torch.Tensor, workspace: torch.Tensor,
+                unique_rows: Optional[torch.Tensor] = None, counts: Optional[torch.Tensor] = None,
+                result: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Enqueue ``dst_densify`` (include/dst.h) for one IndexedSlices gradient."""
+    lib = load_library()
+    _check_slice(indices, values, d, out.device)
+    if out.numel() != vocab * d or not out.is_contiguous():
+        raise ValueError("out must be contiguous [vocab, d]")
+    if dense_in is not None and (dense_in.dtype != out.dtype or dense_in.numel() != vocab * d
+                                 or not dense_in.is_contiguous()):
+        raise ValueError("dense_in must be contiguous [vocab, d] in out's dtype")
+    o = _opts(indices.dtype, values.dtype, out.dtype)
+    with torch.cuda.device(out.device):
+        rc = lib.dst_densify(_ptr(indices), _ptr(values), indices.shape[0], d, vocab, _ptr(dense_in), _ptr(out),
+                             _stream_handle(stream), ctypes.byref(o), _ptr(workspace),
+                             workspace.numel() * workspace.element_size(), _ptr(unique_rows), _ptr(counts),
+                             _ptr(result))
+    if rc != 0:
+        raise DstError(rc, "dst_densify")
+
+
+def dst_densify_concat_host(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]], d: int, vocab: int,
+                            host_dense_in: Optional[torch.Tensor], host_out: torch.Tensor, staging: torch.Tensor,
+                            workspace: torch.Tensor, host_result: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Enqueue ``dst_densify_concat_host``: slices, dense_in and out are HOST (ideally pinned) tensors;
+    ``staging`` and ``workspace`` are CUDA tensors.  host_out is valid after the stream has drained."""
+    lib = load_library()
+    R = len(slices)
+    if R == 0:
+        raise ValueError("need at least one slice")
+    index_dtype, value_dtype = slices[0][0].dtype, slices[0][1].dtype
+    arr = (_Slice * R)()
+    for r, (idx, val) in enumerate(slices):
+        if idx.is_cuda or val.is_cuda:
+            raise ValueError("host entry point: slices must be CPU tensors")
+        if idx.dtype != index_dtype or val.dtype != value_dtype:
+            raise TypeError("all slices must share index and value dtypes")
+        _check_slice(idx, val, d, torch.device("cpu"))
+        arr[r].indices, arr[r].values, arr[r].n_rows = idx.data_ptr(), val.data_ptr(), idx.shape[0]
+    o = _opts(index_dtype, value_dtype, host_out.dtype)
+    with torch.cuda.device(staging.device):
+        rc = lib.dst_densify_concat_host(arr, R, d, vocab, _ptr(host_dense_in), _ptr(host_out),
+                                         _stream_handle(stream), ctypes.byref(o), _ptr(staging),
+                                         staging.numel() * staging.element_size(), _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _ptr(host_result))
+    if rc != 0:
+        raise DstError(rc, "dst_densify_concat_host")
+
+
+class Densifier:
+    """Owns the caller-side buffers (workspace, result block, optional unique/count arrays) for
+    repeated calls on one shape; the arithmetic stays in the library."""
+
+    def __init__(self, n_rows_total: int, R: int, d: int, vocab: int, *, index_dtype=torch.int64,
+                 value_dtype=torch.float32, out_dtype=torch.float32, device="cuda", want_unique: bool = True):
+        self.n_rows_total, self.R, self.d, self.vocab = n_rows_total, R, d, vocab
+        self.index_dtype, self.value_dtype, self.out_dtype = index_dtype, value_dtype, out_dtype
+        self.device = torch.device(device)
+        nbytes = dst_workspace_bytes(n_rows_total, R, d, vocab, index_dtype, value_dtype, out_dtype)
+        if nbytes == 0 and vocab and d:
+            raise DstError(2, "dst_workspace_bytes")
+        self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=self.device)
+        self.result = torch.zeros(RESULT_BYTES // 4, dtype=torch.int32, device=self.device)
+        cap = max(1, min(n_rows_total, vocab))
+        self.unique_rows = torch.empty(cap, dtype=index_dtype, device=self.device) if want_unique else None
+        self.counts = torch.empty(cap, dtype=torch.int32, device=self.device) if want_unique else None
+
+    def __call__(self, slices, dense_in, out, stream=None):
+        dst_densify_concat(slices, self.d, self.vocab, dense_in, out, self.workspace, self.unique_rows,
+                           self.counts, self.result, stream, self.index_dtype, self.value_dtype)
+        return out
+
+    def densify(self, indices, values, dense_in, out, stream=None):
+        dst_densify(indices, values, self.d, self.vocab, dense_in, out, self.workspace, self.unique_rows,
+                    self.counts, self.result, stream)
+        return out
+
+    def read_result(self) -> dict:
+        """Synchronising read of the dst_result_t the last call wrote."""
+        raw = self.result.cpu().numpy().tobytes()
+        r = _Result.from_buffer_copy(raw)
+        return {"status": r.status, "n_unique": r.n_unique, "n_out_of_range": r.n_out_of_range,
+                "max_segment": r.max_segment}

@@ -1,0 +1,260 @@
+// C ABI of the densify library: argument checks, workspace carving, kernel sequencing.
+#include <string.h>
+
+#include <atomic>
+
+#include "dst_common.cuh"
+
+namespace dst {
+
+static thread_local cudaEvent_t t_ev_before = nullptr, t_ev_after = nullptr;
+static std::atomic<long long> g_launches{0};
+
+static size_t index_size(int t) { return t == DST_I64 ? 8 : 4; }
+static size_t dtype_size(int t) { return t == DST_F32 ? 4 : 2; }
+
+static bool opts_ok(const dst_opts_t* o) {
+    return o && (o->index_type == DST_I32 || o->index_type == DST_I64) &&
+           (o->value_type == DST_F32 || o->value_type == DST_BF16) &&
+           (o->out_type == DST_F32 || o->out_type == DST_BF16) && o->flags == 0;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int sm_count() {
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            cached = n;
+        else
+            return kSmCount;
+    }
+    return cached;
+}
+
+static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
+                        void* out, cudaStream_t stream, const dst_opts_t* opts, void* workspace,
+                        size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
+    if (!opts_ok(opts)) return opts ? DST_ERR_UNSUPPORTED : DST_ERR_INVALID_ARG;
+    if (R < 0 || d < 0 || vocab < 0 || (R > 0 && !slices)) return DST_ERR_INVALID_ARG;
+    if (vocab > kMaxVocab) return DST_ERR_UNSUPPORTED;
+    int64_t n_total = 0;
+    for (int r = 0; r < R; ++r) {
+        if (slices[r].n_rows < 0) return DST_ERR_INVALID_ARG;
+        if (slices[r].n_rows > 0 && (!slices[r].indices || (!slices[r].values && d > 0))) return DST_ERR_INVALID_ARG;
+        n_total += slices[r].n_rows;
+        if (n_total > kMaxRows) return DST_ERR_UNSUPPORTED;
+    }
+    if (vocab == 0 || d == 0) return DST_OK;
+    if (!out || !workspace) return DST_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return DST_ERR_INVALID_ARG;
+    const Layout L = make_layout(n_total, R, d, vocab);
+    if (workspace_bytes < L.total) return DST_ERR_WORKSPACE_TOO_SMALL;
+
+    char* ws = static_cast<char*>(workspace);
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(ws + L.off_header);
+    unsigned* count = reinterpret_cast<unsigned*>(ws + L.off_count);
+    unsigned* digit = reinterpret_cast<unsigned*>(ws + L.off_digit);
+    unsigned* desc = reinterpret_cast<unsigned*>(ws + L.off_desc);
+    unsigned* nodecnt = reinterpret_cast<unsigned*>(ws + L.off_nodecnt);
+    int* offsets = reinterpret_cast<int*>(ws + L.off_offsets);
+    unsigned* keys[2] = {reinterpret_cast<unsigned*>(ws + L.off_keys[0]), reinterpret_cast<unsigned*>(ws + L.off_keys[1])};
+    unsigned* pos[2] = {reinterpret_cast<unsigned*>(ws + L.off_pos[0]), reinterpret_cast<unsigned*>(ws + L.off_pos[1])};
+    SliceEntry* tab = reinterpret_cast<SliceEntry*>(ws + L.off_tab);
+    HeavyInfo* heavy = reinterpret_cast<HeavyInfo*>(ws + L.off_heavy);
+    ChunkDesc* chunkdesc = reinterpret_cast<ChunkDesc*>(ws + L.off_chunkdesc);
+    float* partials = reinterpret_cast<float*>(ws + L.off_partials);
+
+    // the fast kernels need 16-byte aligned rows everywhere
+    const int vc = int(16 / dtype_size(opts->value_type));
+    bool vector_ok = d % vc == 0 && aligned16(out) && aligned16(dense_in);
+    for (int r = 0; r < R && vector_ok; ++r)
+        if (slices[r].n_rows > 0 && !aligned16(slices[r].values)) vector_ok = false;
+
+    if (cudaMemsetAsync(ws, 0, L.zero_bytes, stream) != cudaSuccess) return DST_ERR_CUDA;
+
+    // a1/a2: histogram, at most kHistSlices slices per launch
+    int64_t start = 0;
+    for (int first = 0; first < R; first += kHistSlices) {
+        HistParams P;
+        memset(&P, 0, sizeof P);
+        P.n = R - first < kHistSlices ? R - first : kHistSlices;
+        P.first = first;
+        int64_t longest = 0;
+        for (int i = 0; i < P.n; ++i) {
+            const dst_slice_t& s = slices[first + i];
+            P.s[i] = SliceEntry{s.indices, s.values, (long long)start, (long long)s.n_rows};
+            start += s.n_rows;
+            if (s.n_rows > longest) longest = s.n_rows;
+        }
+        int grid_x = int((longest + kTile - 1) / kTile);
+        if (grid_x < 1) grid_x = 1;   // still writes the slice table
+        if (launch_hist(P, grid_x, opts->index_type, hdr, count, digit, keys[0], tab, vocab, L.passes, stream) != cudaSuccess)
+            return DST_ERR_CUDA;
+        ++g_launches;
+    }
+    // a3/a5/a6
+    if (launch_scan(opts->index_type, hdr, count, offsets, heavy, chunkdesc, unique_rows, counts, result,
+                    int(L.vocab_pad), L.chunk, stream) != cudaSuccess)
+        return DST_ERR_CUDA;
+    ++g_launches;
+    // a4: least significant digit first; keys/positions ping-pong between two buffers
+    if (n_total > 0) {
+        for (int p = 0; p < L.passes; ++p) {
+            const bool last = p == L.passes - 1;
+            if (launch_radix_pass(int(L.n_tiles), hdr, keys[p & 1], p == 0 ? nullptr : pos[p & 1],
+                                  last ? nullptr : keys[(p + 1) & 1], pos[(p + 1) & 1], digit + p * 256,
+                                  desc + size_t(p) * size_t(L.n_tiles) * 256, p, int(n_total), stream) != cudaSuccess)
+                return DST_ERR_CUDA;
+            ++g_launches;
+        }
+    }
+    // a7/a8
+    MainArgs a;
+    a.hdr = hdr; a.offsets = offsets; a.perm = pos[L.passes & 1]; a.tab = tab; a.heavy = heavy;
+    a.chunkdesc = chunkdesc; a.node_cnt = nodecnt; a.partials = partials; a.dense_in = dense_in; a.out = out;
+    a.result = result; a.d = d; a.vocab = int(vocab); a.n_total = int(n_total); a.R = R; a.chunk = L.chunk;
+    a.chunk_max = int(L.chunk_max);
+    if (t_ev_before && cudaEventRecord(t_ev_before, stream) != cudaSuccess) return DST_ERR_CUDA;
+    if (launch_reduce_rows(a, opts->value_type, opts->out_type, vector_ok, sm_count() * 4, stream) != cudaSuccess)
+        return DST_ERR_CUDA;
+    ++g_launches;
+    if (t_ev_after && cudaEventRecord(t_ev_after, stream) != cudaSuccess) return DST_ERR_CUDA;
+    return DST_OK;
+}
+
+}  // namespace dst
+
+using namespace dst;
+
+extern "C" {
+
+int dst_version(void) { return 100; }
+
+void dst_profile_events(void* before, void* after) {
+    t_ev_before = static_cast<cudaEvent_t>(before);
+    t_ev_after = static_cast<cudaEvent_t>(after);
+}
+
+int64_t dst_kernel_launches(void) { return g_launches.load(); }
+
+const char* dst_status_string(int status) {
+    switch (status) {
+        case DST_OK: return "ok";
+        case DST_ERR_INVALID_ARG: return "invalid argument";
+        case DST_ERR_UNSUPPORTED: return "unsupported type or size";
+        case DST_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case DST_ERR_INDEX_OUT_OF_RANGE: return "some indices were outside [0, vocab) and were skipped";
+        case DST_ERR_TIMEOUT: return "a bounded device-side wait gave up; output invalid";
+        case DST_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown status";
+    }
+}
+
+size_t dst_workspace_bytes(int64_t n_rows_total, int32_t R, int64_t d, int64_t vocab, const dst_opts_t* opts) {
+    if (!opts_ok(opts) || n_rows_total < 0 || n_rows_total > kMaxRows || R < 0 || d < 0 || vocab < 0 || vocab > kMaxVocab)
+        return 0;
+    return make_layout(n_rows_total, R, d, vocab).total;
+}
+
+int dst_densify(const void* indices, const void* values, int64_t n_rows, int64_t d, int64_t vocab,
+                const void* dense_in, void* out, dst_stream_t stream, const dst_opts_t* opts, void* workspace,
+                size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
+    dst_slice_t s{indices, values, n_rows};
+    return densify_impl(&s, 1, d, vocab, dense_in, out, stream, opts, workspace, workspace_bytes, unique_rows,
+                        counts, result);
+}
+
+int dst_densify_concat(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
+                       void* out, dst_stream_t stream, const dst_opts_t* opts, void* workspace,
+                       size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
+    return densify_impl(slices, R, d, vocab, dense_in, out, stream, opts, workspace, workspace_bytes, unique_rows,
+                        counts, result);
+}
+
+size_t dst_host_staging_bytes(int64_t n_rows_total, int64_t d, int64_t vocab, const dst_opts_t* opts) {
+    if (!opts_ok(opts) || n_rows_total < 0 || d < 0 || vocab < 0) return 0;
+    size_t o = 0;
+    o = align_up(o + size_t(n_rows_total) * index_size(opts->index_type), 256);
+    o = align_up(o + size_t(n_rows_total) * size_t(d) * dtype_size(opts->value_type), 256);
+    o = align_up(o + size_t(vocab) * size_t(d) * dtype_size(opts->out_type), 256);
+    o = align_up(o + sizeof(dst_result_t), 256);
+    return o;
+}
+
+int dst_densify_concat_host(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab,
+                            const void* host_dense_in, void* host_out, dst_stream_t stream, const dst_opts_t* opts,
+                            void* staging, size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                            dst_result_t* host_result) {
+    if (!opts_ok(opts)) return opts ? DST_ERR_UNSUPPORTED : DST_ERR_INVALID_ARG;
+    if (R < 0 || d < 0 || vocab < 0 || (R > 0 && !slices)) return DST_ERR_INVALID_ARG;
+    int64_t n_total = 0;
+    for (int r = 0; r < R; ++r) {
+        if (slices[r].n_rows < 0) return DST_ERR_INVALID_ARG;
+        if (slices[r].n_rows > 0 && (!slices[r].indices || (!slices[r].values && d > 0))) return DST_ERR_INVALID_ARG;
+        n_total += slices[r].n_rows;
+        if (n_total > kMaxRows) return DST_ERR_UNSUPPORTED;
+    }
+    if (vocab == 0 || d == 0) return DST_OK;
+    if (!host_out || !staging || (reinterpret_cast<uintptr_t>(staging) & 255u)) return DST_ERR_INVALID_ARG;
+    if (staging_bytes < dst_host_staging_bytes(n_total, d, vocab, opts)) return DST_ERR_WORKSPACE_TOO_SMALL;
+    if (!workspace || workspace_bytes < dst_workspace_bytes(n_total, 1, d, vocab, opts)) return DST_ERR_WORKSPACE_TOO_SMALL;
+    const size_t si = index_size(opts->index_type), sv = dtype_size(opts->value_type), so = dtype_size(opts->out_type);
+    char* st = static_cast<char*>(staging);
+    size_t o = 0;
+    char* d_idx = st + o; o = align_up(o + size_t(n_total) * si, 256);
+    char* d_val = st + o; o = align_up(o + size_t(n_total) * size_t(d) * sv, 256);
+    char* d_out = st + o; o = align_up(o + size_t(vocab) * size_t(d) * so, 256);
+    dst_result_t* d_res = reinterpret_cast<dst_result_t*>(st + o);
+    // host -> device: the slices land back to back, i.e. as their concatenation
+    size_t row = 0;
+    for (int r = 0; r < R; ++r) {
+        const size_t n = size_t(slices[r].n_rows);
+        if (n == 0) continue;
+        if (cudaMemcpyAsync(d_idx + row * si, slices[r].indices, n * si, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+            cudaMemcpyAsync(d_val + row * size_t(d) * sv, slices[r].values, n * size_t(d) * sv, cudaMemcpyHostToDevice,
+                            stream) != cudaSuccess)
+            return DST_ERR_CUDA;
+        row += n;
+    }
+    const size_t out_bytes = size_t(vocab) * size_t(d) * so;
+    if (host_dense_in &&
+        cudaMemcpyAsync(d_out, host_dense_in, out_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return DST_ERR_CUDA;
+    dst_slice_t s{d_idx, d_val, n_total};
+    int rc = densify_impl(&s, 1, d, vocab, host_dense_in ? d_out : nullptr, d_out, stream, opts, workspace,
+                          workspace_bytes, nullptr, nullptr, d_res);
+    if (rc != DST_OK) return rc;
+    if (cudaMemcpyAsync(host_out, d_out, out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return DST_ERR_CUDA;
+    if (host_result &&
+        cudaMemcpyAsync(host_result, d_res, sizeof(dst_result_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return DST_ERR_CUDA;
+    return DST_OK;
+}
+
+int dst_bytes_report(const int64_t* n_rows_per_slice, int32_t R, int64_t d, int64_t vocab, const dst_opts_t* opts,
+                     dst_bytes_report_t* report) {
+    if (!opts_ok(opts)) return opts ? DST_ERR_UNSUPPORTED : DST_ERR_INVALID_ARG;
+    if (!report || R < 0 || d < 0 || vocab < 0 || (R > 0 && !n_rows_per_slice)) return DST_ERR_INVALID_ARG;
+    const int64_t si = int64_t(index_size(opts->index_type)), sv = int64_t(dtype_size(opts->value_type)),
+                  so = int64_t(dtype_size(opts->out_type));
+    int64_t n_total = 0, gather_all = 0;
+    for (int r = 0; r < R; ++r) {
+        if (n_rows_per_slice[r] < 0) return DST_ERR_INVALID_ARG;
+        n_total += n_rows_per_slice[r];
+        gather_all += (vocab + n_rows_per_slice[r]) * d * sv;
+    }
+    report->n_rows_total = n_total;
+    report->sparse_value_bytes = n_total * d * sv;
+    report->sparse_index_bytes = n_total * si;
+    report->sparse_bytes = report->sparse_value_bytes + report->sparse_index_bytes;
+    report->dense_bytes = vocab * d * so;
+    report->gather_all_value_bytes = gather_all;
+    report->sparse_over_dense = report->dense_bytes ? double(report->sparse_bytes) / double(report->dense_bytes) : 0.0;
+    report->gather_all_over_dense = report->dense_bytes ? double(gather_all) / double(report->dense_bytes) : 0.0;
+    return DST_OK;
+}
+
+}  // extern "C"

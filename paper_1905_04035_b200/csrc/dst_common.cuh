@@ -1,0 +1,176 @@
+// Shared definitions for the densify kernels: workspace layout, small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dst.h"
+
+namespace dst {
+
+// ---- fixed shape parameters -------------------------------------------------
+constexpr int kSortThreads = 256;           // threads of the histogram and radix-pass kernels
+constexpr int kSortItems = 8;               // keys per thread
+constexpr int kTile = kSortThreads * kSortItems;  // 2048 keys per CTA
+constexpr int kHashSlots = 4096;            // per-CTA key aggregation table (> kTile distinct keys never happen)
+constexpr int kMaxPasses = 4;               // 8-bit digits, keys below 2^31
+constexpr int kFanIn = 16;                  // children per node of the heavy-row combine tree
+constexpr int kRowsPerBatch = 4;            // output rows per light work item
+constexpr int kMainThreads = 256;
+constexpr int kScanThreads = 1024;
+constexpr int kScanItems = 16;              // counters per thread and round in the scan kernel
+constexpr int kSmCount = 148;               // B200; only used to pick the chunk length
+constexpr unsigned kInvalidKey = 0xFFFFFFFFu;
+constexpr unsigned kFlagMask = 0xC0000000u, kFlagAggregate = 0x40000000u, kFlagPrefix = 0x80000000u;
+constexpr unsigned kValueMask = 0x3FFFFFFFu;
+constexpr int64_t kMaxRows = (int64_t(1) << 30) - 1;  // look-back words keep 30 bits of count
+constexpr int64_t kMaxVocab = int64_t(1) << 30;
+constexpr int kSpinLimit = 1 << 20;
+
+// ---- workspace --------------------------------------------------------------
+struct WsHeader {          // zeroed at the start of every call
+    int status;            // device-detected dst_status_t (max wins)
+    int n_valid;           // rows with an index inside [0, vocab)
+    int n_unique;
+    int n_heavy;           // rows with more than `chunk` occurrences
+    int n_chunks;          // work items those rows are split into
+    int n_upper;           // combine-tree nodes above the chunk level
+    int max_segment;
+    int pad0;
+    unsigned long long n_bad;
+    unsigned int ticket[kMaxPasses];
+    unsigned int work_counter;
+    unsigned int pad1[3];
+};
+static_assert(sizeof(WsHeader) == 72, "header layout");
+
+struct SliceEntry {        // one IndexedSlices object of the (virtual) concatenation
+    const void* indices;
+    const void* values;
+    long long start;       // global position of its first row
+    long long n_rows;
+};
+
+constexpr int kHistSlices = 64;   // slices described per histogram launch (kernel-parameter space)
+struct HistParams {
+    SliceEntry s[kHistSlices];
+    int n;                 // slices used in this launch
+    int first;             // index of s[0] in the full slice table
+};
+
+struct HeavyInfo {         // a row whose segment is split into chunks
+    int row;
+    int chunk_base;        // id of its first chunk
+    int upper_base;        // id of its first upper tree node
+    int n_chunks;
+};
+
+struct ChunkDesc {         // one chunk work item
+    int row;
+    int begin;             // first entry in perm[]
+    int len;
+    int heavy;             // index into HeavyInfo
+};
+
+struct Layout {
+    int64_t n_rows, vocab, d;
+    int R, chunk, passes;
+    int64_t n_tiles, vocab_pad, heavy_max, chunk_max, upper_max;
+    size_t off_header, off_count, off_digit, off_desc, off_nodecnt, zero_bytes;
+    size_t off_offsets, off_keys[2], off_pos[2], off_tab, off_heavy, off_chunkdesc, off_partials;
+    size_t total;
+};
+
+// arguments of the row-reduction kernels
+struct MainArgs {
+    WsHeader* hdr;
+    const int* offsets;
+    const unsigned* perm;
+    const SliceEntry* tab;
+    const HeavyInfo* heavy;
+    const ChunkDesc* chunkdesc;
+    unsigned* node_cnt;
+    float* partials;
+    const void* dense_in;
+    void* out;
+    dst_result_t* result;
+    long long d;
+    int vocab;
+    int n_total;     // rows in all slices (capacity of perm)
+    int R;
+    int chunk;
+    int chunk_max;   // partial rows of the chunk level; upper nodes follow
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Everything about the workspace follows from the shapes alone, so the same
+// shapes always give the same chunking and therefore the same summation order.
+inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab) {
+    Layout L{};
+    L.n_rows = n_rows; L.vocab = vocab; L.d = d; L.R = R;
+    // chunk length: keep work items near 1/32 of an SM's fair share of rows
+    int64_t units = 2 * vocab + n_rows;
+    int64_t per = units / (int64_t(kSmCount) * 32);
+    int c = 16;
+    while (c < 256 && c * 2 <= per) c *= 2;
+    L.chunk = c;
+    int bits = 0;
+    while (bits < 31 && (int64_t(1) << bits) < vocab) ++bits;   // keys are < vocab <= 2^bits
+    L.passes = bits <= 8 ? 1 : (bits + 7) / 8;
+    L.n_tiles = (n_rows + kTile - 1) / kTile;
+    L.vocab_pad = (vocab + kScanItems - 1) / kScanItems * kScanItems;
+    L.heavy_max = n_rows / (c + 1);
+    L.chunk_max = n_rows / c + L.heavy_max;
+    L.upper_max = L.chunk_max / 2 + L.heavy_max + 1;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    L.off_header = take(sizeof(WsHeader));
+    L.off_count = take(size_t(L.vocab_pad) * 4);
+    L.off_digit = take(size_t(kMaxPasses) * 256 * 4);
+    L.off_desc = take(size_t(L.passes) * size_t(L.n_tiles) * 256 * 4);
+    L.off_nodecnt = take(size_t(L.upper_max) * 4);
+    L.zero_bytes = o;
+    L.off_offsets = take(size_t(L.vocab_pad + kScanItems) * 4);
+    L.off_keys[0] = take(size_t(n_rows) * 4);
+    L.off_keys[1] = take(size_t(n_rows) * 4);
+    L.off_pos[0] = take(size_t(n_rows) * 4);
+    L.off_pos[1] = take(size_t(n_rows) * 4);
+    L.off_tab = take(size_t(R > 0 ? R : 1) * sizeof(SliceEntry));
+    L.off_heavy = take(size_t(L.heavy_max + 1) * sizeof(HeavyInfo));
+    L.off_chunkdesc = take(size_t(L.chunk_max + 1) * sizeof(ChunkDesc));
+    L.off_partials = take(size_t(L.chunk_max + L.upper_max) * size_t(d) * 4);
+    L.total = o;
+    return L;
+}
+
+// ---- kernel launchers (defined next to their kernels) ----------------------------
+cudaError_t launch_hist(const HistParams& P, int grid_x, int index_type, WsHeader* hdr, unsigned* count,
+                        unsigned* digit_hist, unsigned* keys, SliceEntry* tab, long long vocab, int passes,
+                        cudaStream_t stream);
+cudaError_t launch_scan(int index_type, WsHeader* hdr, const unsigned* count, int* offsets, HeavyInfo* heavy,
+                        ChunkDesc* chunkdesc, void* unique_rows, int* counts_out, dst_result_t* result,
+                        int vocab_pad, int chunk, cudaStream_t stream);
+cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
+                              unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
+                              int pass, int capacity, cudaStream_t stream);
+cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int grid,
+                               cudaStream_t stream);
+
+// ---- device helpers ---------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
+__device__ __forceinline__ int warp_id() { return threadIdx.x >> 5; }
+
+__device__ __forceinline__ void raise_status(WsHeader* hdr, int code) { atomicMax(&hdr->status, code); }
+
+// Number of combine-tree nodes above the chunk level for a row split into n chunks.
+__host__ __device__ __forceinline__ int upper_nodes(int n) {
+    int u = 0;
+    while (n > 1) { n = (n + kFanIn - 1) / kFanIn; u += n; }
+    return u;
+}
+#endif
+
+}  // namespace dst
