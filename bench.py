@@ -1,0 +1,423 @@
+#!/usr/bin/env python
+"""Benchmark of the densify hot path: GB/s and rows/s on B200, fraction of the HBM roofline,
+the CPU oracle beside it.
+
+One "step" is one pass of the whole hot path (index histogram, scan, radix placement, row
+reduction with the fused dense add) over one batch of synthetic IndexedSlices.  The headline
+workload is the R=64 concatenated-slices configuration (the largest of the configurations,
+2.7 GB of value rows, far larger than L2); the other configurations are reported in
+"all_configs" of the same JSON line.
+
+  python bench.py                       # 1 GPU, headline + all configurations + CPU oracle baseline
+  python bench.py --workload big        # another headline workload
+  python bench.py --impl reference      # the CPU oracle as the reference arm
+  torchrun ... bench.py --gpus N        # N independent replicas (the path has no exchange step)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1905_04035_b200.workloads import make_workload  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+SIZEOF = {"f32": 4, "bf16": 2, "i32": 4, "i64": 8}
+FALLBACK_HBM_GBS = 6650.0
+ALL_CONFIGS = ("tiny", "base", "big", "r64", "sweep_uniform", "sweep_zipf", "sweep_same")
+
+
+def algorithmic_bytes(w) -> int:
+    """Values read once + dense_in read once + out written once + indices read once."""
+    n = w.n_rows_total
+    b = n * w.d * SIZEOF[w.value_dtype] + w.vocab * w.d * SIZEOF[w.out_dtype] + n * SIZEOF[w.index_dtype]
+    if w.dense_in is not None:
+        b += w.vocab * w.d * SIZEOF[w.out_dtype]
+    return b
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="dst_clocks_", suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return None
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); smax.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if not sm:
+            return None
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------------------------
+def _dev_tensor(arr, kind, device):
+    import torch
+    if kind == "bf16":
+        return torch.from_numpy(arr.view(np.int16)).to(device).view(torch.bfloat16)
+    return torch.from_numpy(arr).to(device)
+
+
+class DeviceProblem:
+    """A workload resident in HBM, with enough rotating copies that consecutive steps never
+    find their inputs in L2."""
+
+    def __init__(self, w, device, n_sets=None):
+        import torch
+        import paper_1905_04035_b200 as dst
+        self.w, self.device = w, device
+        tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "i32": torch.int32, "i64": torch.int64}
+        self.balg = algorithmic_bytes(w)
+        if n_sets is None:
+            n_sets = 1 if self.balg >= 4 * L2_BYTES else int(min(8, -(-4 * L2_BYTES // max(self.balg, 1))))
+        self.n_sets = n_sets
+        self.sets = []
+        for _ in range(n_sets):
+            slices = [(_dev_tensor(i, w.index_dtype, device), _dev_tensor(v, w.value_dtype, device))
+                      for i, v in zip(w.indices, w.values)]
+            dense = _dev_tensor(w.dense_in, w.out_dtype, device) if w.dense_in is not None else None
+            out = torch.empty(w.vocab, w.d, dtype=tdt[w.out_dtype], device=device)
+            self.sets.append((slices, dense, out))
+        self.eng = dst.Densifier(w.n_rows_total, w.R, w.d, w.vocab, index_dtype=tdt[w.index_dtype],
+                                 value_dtype=tdt[w.value_dtype], out_dtype=tdt[w.out_dtype], device=device,
+                                 want_unique=True)
+        self.flush = None
+        if n_sets * self.balg < 4 * L2_BYTES:
+            self.flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+
+    def step(self, k: int):
+        slices, dense, out = self.sets[k % self.n_sets]
+        self.eng(slices, dense, out)
+
+    def l2_policy(self) -> str:
+        if self.n_sets == 1 and self.flush is None:
+            return "inputs larger than L2 (%.0f MB per step vs 126 MB L2)" % (self.balg / 1e6)
+        if self.flush is None:
+            return "rotating %d buffer sets (%.0f MB total) so no step finds its inputs in L2" % (
+                self.n_sets, self.n_sets * self.balg / 1e6)
+        return "L2 flushed by a 252 MB write between steps"
+
+
+def time_device(prob: DeviceProblem, steps: int, warmup: int, dist_ctx=None, clocks: ClockSampler = None):
+    """K steps bracketed by sync (+ barrier); returns (total ms, per-step reduce-kernel ms list, launches)."""
+    import torch
+    import paper_1905_04035_b200 as dst
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in kev:
+        a.record(); b.record()        # creates the underlying CUDA events
+    for k in range(warmup):
+        if prob.flush is not None:
+            prob.flush.zero_()
+        prob.step(k)
+    torch.cuda.synchronize()
+    if dist_ctx is not None:
+        dist_ctx.barrier()
+    if clocks is not None:
+        clocks.start()
+    launches0 = dst.dst_kernel_launches()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_ev = []
+    torch.cuda.synchronize()
+    if prob.flush is None:
+        t0.record()
+        for k in range(steps):
+            dst.dst_profile_events(*kev[k])
+            prob.step(warmup + k)
+        t1.record()
+        torch.cuda.synchronize()
+        total_ms = t0.elapsed_time(t1)
+    else:
+        # the flush is not part of the step: time each step on its own and add them up
+        for k in range(steps):
+            prob.flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            dst.dst_profile_events(*kev[k])
+            a.record(); prob.step(warmup + k); b.record()
+            step_ev.append((a, b))
+        torch.cuda.synchronize()
+        total_ms = float(sum(a.elapsed_time(b) for a, b in step_ev))
+    dst.dst_profile_events(None, None)
+    launches = dst.dst_kernel_launches() - launches0
+    clock_info = clocks.stop() if clocks is not None else None
+    if dist_ctx is not None:
+        dist_ctx.barrier()
+    kernel_ms = [a.elapsed_time(b) for a, b in kev]
+    return total_ms, kernel_ms, launches, clock_info
+
+
+def time_e2e(w, device, steps: int, warmup: int):
+    """Same metric through the host entry point: pinned host buffers, H2D and D2H inside the timed region."""
+    import torch
+    import paper_1905_04035_b200 as dst
+    tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "i32": torch.int32, "i64": torch.int64}
+
+    def host(arr, kind):
+        t = torch.from_numpy(arr.view(np.int16)).view(torch.bfloat16) if kind == "bf16" else torch.from_numpy(arr)
+        return t.pin_memory()
+
+    slices = [(host(i, w.index_dtype), host(v, w.value_dtype)) for i, v in zip(w.indices, w.values)]
+    dense = host(w.dense_in, w.out_dtype) if w.dense_in is not None else None
+    out = torch.empty(w.vocab, w.d, dtype=tdt[w.out_dtype]).pin_memory()
+    res = torch.zeros(6, dtype=torch.int32).pin_memory()
+    n = w.n_rows_total
+    staging = torch.empty(dst.dst_host_staging_bytes(n, w.d, w.vocab, tdt[w.index_dtype], tdt[w.value_dtype],
+                                                     tdt[w.out_dtype]), dtype=torch.uint8, device=device)
+    ws = torch.empty(dst.dst_workspace_bytes(n, 1, w.d, w.vocab, tdt[w.index_dtype], tdt[w.value_dtype],
+                                             tdt[w.out_dtype]), dtype=torch.uint8, device=device)
+    for _ in range(warmup):
+        dst.dst_densify_concat_host(slices, w.d, w.vocab, dense, out, staging, ws, res)
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        dst.dst_densify_concat_host(slices, w.d, w.vocab, dense, out, staging, ws, res)
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / steps
+    h2d = n * (w.d * SIZEOF[w.value_dtype] + SIZEOF[w.index_dtype]) + (out.numel() * out.element_size() if dense is not None else 0)
+    d2h = out.numel() * out.element_size() + 24
+    assert res[0].item() == 0
+    return ms, int(h2d), int(d2h)
+
+
+# ---------------------------------------------------------------------------------------------
+# the CPU oracle arm (reference arm and cpu_baseline leg)
+# ---------------------------------------------------------------------------------------------
+def time_oracle(w, max_rows=None, repeats=1):
+    """Time the oracle as it stands on (a prefix of every slice of) the workload.  Single thread."""
+    import oracle
+    idx, val = w.indices, w.values
+    sample = "full workload"
+    if max_rows is not None and w.n_rows_total > max_rows:
+        keep = max(1, max_rows // max(w.R, 1))
+        idx = [i[:keep] for i in idx]
+        val = [v[:keep] for v in val]
+        sample = "first %d rows of each of the %d slices (%d of %d rows), full [vocab, d] dense add and output" % (
+            keep, w.R, keep * w.R, w.n_rows_total)
+    n = int(sum(i.shape[0] for i in idx))
+    best = None
+    for _ in range(repeats):
+        t = time.perf_counter()
+        oracle.densify(idx, val, w.d, w.vocab, w.dense_in, value_dtype=w.value_dtype, out_dtype=w.out_dtype)
+        dt = time.perf_counter() - t
+        best = dt if best is None else min(best, dt)
+    b = n * w.d * SIZEOF[w.value_dtype] + w.vocab * w.d * SIZEOF[w.out_dtype] + n * SIZEOF[w.index_dtype]
+    if w.dense_in is not None:
+        b += w.vocab * w.d * SIZEOF[w.out_dtype]
+    return {"seconds": best, "rows": n, "bytes": b, "gbs": b / best / 1e9, "rows_per_s": n / best, "sample": sample}
+
+
+# ---------------------------------------------------------------------------------------------
+def run_config(name, device, steps, warmup, seed, dist_ctx=None, clocks=None, want_e2e=False, e2e_steps=5):
+    import torch
+    peak, peak_src = measured_peak()
+    w = make_workload(name, seed=seed)
+    prob = DeviceProblem(w, device)
+    total_ms, kernel_ms, launches, clock_info = time_device(prob, steps, warmup, dist_ctx, clocks)
+    res = prob.eng.read_result()
+    ms = total_ms / steps
+    kms = float(np.mean(kernel_ms))
+    out = {
+        "workload": name, "ms_per_step": ms, "gbs": prob.balg / ms / 1e6, "rows_per_s": w.n_rows_total / ms * 1e3,
+        "frac_of_hbm_peak": prob.balg / ms / 1e6 / peak, "algorithmic_bytes": prob.balg,
+        "reduce_kernel_ms": kms, "reduce_kernel_gbs": prob.balg / kms / 1e6,
+        "reduce_kernel_frac": prob.balg / kms / 1e6 / peak, "launches": launches, "l2": prob.l2_policy(),
+        "n_unique": res["n_unique"], "max_segment": res["max_segment"], "status": res["status"],
+        "peak_gbs": peak, "peak_source": peak_src, "clocks": clock_info, "w": w,
+    }
+    del prob
+    torch.cuda.empty_cache()
+    if want_e2e:
+        ems, h2d, d2h = time_e2e(w, device, e2e_steps, 2)
+        out["e2e"] = {"ms_per_step": ems, "gbs": out["algorithmic_bytes"] / ems / 1e6, "h2d": h2d, "d2h": d2h}
+        torch.cuda.empty_cache()
+    return out
+
+
+def reference_arm(args):
+    """The oracle, timed on the host cores, as the reference arm (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = make_workload(args.workload, seed=args.seed)
+    cap = args.reference_rows
+    times = []
+    info = None
+    for k in range(args.warmup + args.steps):
+        info = time_oracle(w, max_rows=cap)
+        if k >= args.warmup:
+            times.append(info["seconds"])
+    sec = float(np.mean(times))
+    gbs = info["bytes"] / sec / 1e9
+    line = {
+        "impl": "reference", "metric": "densify_GBps", "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "recipe": w.recipe, "vocab": w.vocab, "d": w.d, "R": w.R,
+                   "n_rows_total": w.n_rows_total},
+        "rows_per_s": info["rows"] / sec,
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": info["sample"]},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="dst", choices=["dst", "reference"])
+    ap.add_argument("--workload", default="r64", choices=ALL_CONFIGS)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--headline-only", action="store_true", help="skip the other configurations")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--reference-rows", type=int, default=163840,
+                    help="rows of the workload the reference arm processes per step")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "dst" else args.warmup
+
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_1905_04035_b200 as dst
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the densify path")
+    dst.load_library()
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist_ctx = None
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+        dist_ctx = dist
+
+    # every rank is an independent replica with its own seed (the path has no exchange step)
+    from paper_1905_04035_b200.replicas import combine_over_ranks, replica_seed
+    seed = replica_seed(args.seed, rank)
+    clocks = ClockSampler(local_rank) if rank == 0 else None
+    head = run_config(args.workload, device, args.steps, args.warmup, seed, dist_ctx, clocks,
+                      want_e2e=not args.no_e2e)
+    w = head.pop("w")
+
+    agg = combine_over_ranks(head["ms_per_step"], head["algorithmic_bytes"], w.n_rows_total, dist_ctx, device)
+    e2e = None
+    if "e2e" in head:
+        eagg = combine_over_ranks(head["e2e"]["ms_per_step"], head["algorithmic_bytes"], w.n_rows_total, dist_ctx, device)
+        e2e = {"value": eagg["gbs"], "unit": "GB/s", "h2d_bytes_per_step": head["e2e"]["h2d"],
+               "d2h_bytes_per_step": head["e2e"]["d2h"], "ms_per_step": eagg["ms_per_step"]}
+
+    others = []
+    if rank == 0 and world == 1 and not args.headline_only:
+        for name in ALL_CONFIGS:
+            if name == args.workload:
+                continue
+            r = run_config(name, device, min(args.steps, 200), args.warmup, args.seed)
+            r.pop("w"); r.pop("clocks")
+            others.append({k: r[k] for k in ("workload", "ms_per_step", "gbs", "rows_per_s", "frac_of_hbm_peak",
+                                             "algorithmic_bytes", "reduce_kernel_ms", "reduce_kernel_frac", "l2",
+                                             "n_unique", "max_segment", "status")})
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        info = time_oracle(w, max_rows=None if w.n_rows_total <= 700000 else 700000)
+        cpu = {"value": info["gbs"], "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": info["sample"],
+               "seconds": info["seconds"], "rows_per_s": info["rows_per_s"]}
+
+    if rank == 0:
+        rep = dst.dst_bytes_report([int(i.shape[0]) for i in w.indices], w.d, w.vocab,
+                                   *[{"f32": torch.float32, "bf16": torch.bfloat16, "i32": torch.int32,
+                                      "i64": torch.int64}[k] for k in (w.index_dtype, w.value_dtype, w.out_dtype)])
+        line = {
+            "metric": "densify_GBps", "value": agg["gbs"], "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": agg["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32" if w.value_dtype == "f32" else "bf16 in, f32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": args.workload, "recipe": w.recipe, "vocab": w.vocab, "d": w.d, "R": w.R,
+                       "n_rows_total": w.n_rows_total, "l2": head["l2"], "replicas": world},
+            "rows_per_s": agg["rows_per_s"], "frac_of_hbm_peak": agg["gbs"] / world / head["peak_gbs"],
+            "roofline": {"bound": "hbm", "achieved": head["reduce_kernel_gbs"], "peak": head["peak_gbs"],
+                         "unit": "GB/s", "frac": head["reduce_kernel_frac"], "traffic": None,
+                         "kernel": "k_reduce_rows", "of": head["peak_source"],
+                         "kernel_ms": head["reduce_kernel_ms"]},
+            "e2e": e2e, "gpu_launches": head["launches"], "clocks": head["clocks"],
+            "cpu_baseline": cpu, "bytes_report": rep, "all_configs": others,
+            "parity": {"status": head["status"], "n_unique": head["n_unique"], "max_segment": head["max_segment"]},
+        }
+        print(json.dumps(line))
+    if dist_ctx is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
