@@ -270,10 +270,11 @@ def time_oracle(w, max_rows=None, repeats=1):
 
 
 # ---------------------------------------------------------------------------------------------
-def run_config(name, device, steps, warmup, seed, dist_ctx=None, clocks=None, want_e2e=False, e2e_steps=5):
+def run_config(name, device, steps, warmup, seed, dist_ctx=None, clocks=None, want_e2e=False, e2e_steps=5,
+               scale=1.0):
     import torch
     peak, peak_src = measured_peak()
-    w = make_workload(name, seed=seed)
+    w = make_workload(name, seed=seed, scale=scale)
     prob = DeviceProblem(w, device)
     total_ms, kernel_ms, launches, clock_info = time_device(prob, steps, warmup, dist_ctx, clocks)
     res = prob.eng.read_result()
@@ -336,6 +337,8 @@ def main():
     ap.add_argument("--headline-only", action="store_true", help="skip the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--scale", type=float, default=1.0,
+                    help="shrink the rows per slice (profiling captures on a small case); 1.0 = the named configuration")
     ap.add_argument("--reference-rows", type=int, default=163840,
                     help="rows of the workload the reference arm processes per step")
     args = ap.parse_args()
@@ -367,7 +370,7 @@ def main():
     seed = replica_seed(args.seed, rank)
     clocks = ClockSampler(local_rank) if rank == 0 else None
     head = run_config(args.workload, device, args.steps, args.warmup, seed, dist_ctx, clocks,
-                      want_e2e=not args.no_e2e)
+                      want_e2e=not args.no_e2e, scale=args.scale)
     w = head.pop("w")
 
     agg = combine_over_ranks(head["ms_per_step"], head["algorithmic_bytes"], w.n_rows_total, dist_ctx, device)
@@ -404,7 +407,7 @@ def main():
             "vs_baseline": None, "dtype": "f32" if w.value_dtype == "f32" else "bf16 in, f32 accumulate",
             "data": "synthetic",
             "config": {"workload": args.workload, "recipe": w.recipe, "vocab": w.vocab, "d": w.d, "R": w.R,
-                       "n_rows_total": w.n_rows_total, "l2": head["l2"], "replicas": world},
+                       "n_rows_total": w.n_rows_total, "l2": head["l2"], "replicas": world, "scale": args.scale},
             "rows_per_s": agg["rows_per_s"], "frac_of_hbm_peak": agg["gbs"] / world / head["peak_gbs"],
             "roofline": {"bound": "hbm", "achieved": head["reduce_kernel_gbs"], "peak": head["peak_gbs"],
                          "unit": "GB/s", "frac": head["reduce_kernel_frac"], "traffic": None,
