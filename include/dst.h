@@ -130,6 +130,37 @@ int dst_densify_concat(const dst_slice_t* slices, int32_t R, int64_t d, int64_t 
                        void* workspace, size_t workspace_bytes,
                        void* unique_rows, int32_t* counts, dst_result_t* result);
 
+/*
+ * dst_densify without a caller-supplied workspace.  (The paper has no counterpart:
+ * this entry point exists for the sake of callers, not of the method.)
+ *
+ * Who needs it: code that must not, or cannot, obtain device memory at the time it
+ * calls -- a plugin running inside a framework whose allocator it may not re-enter,
+ * a callback on a path where cudaMalloc's implicit device synchronisation is not
+ * acceptable, a process whose memory pool was sized up front and is full.  For those
+ * callers the scratch memory lives inside the library: one array of
+ * DST_STATIC_WORKSPACE_BYTES in device global memory, reserved on every GPU that
+ * loads the library for as long as the process lives.  This call allocates and frees
+ * nothing, on the host side through CUDA or otherwise.
+ *
+ * Arguments, results and summation order are those of dst_densify; the output is
+ * bit-identical to dst_densify on the same inputs.  Differences:
+ *   - Shapes whose workspace need, dst_workspace_bytes(n_rows, 1, d, vocab, opts),
+ *     exceeds DST_STATIC_WORKSPACE_BYTES are refused with
+ *     DST_ERR_WORKSPACE_TOO_SMALL before anything is enqueued.
+ *   - The first call on each device looks up the array's device address (with that
+ *     device current) and keeps it; make that first call outside any stream capture.
+ *     A failure of the look-up is reported as DST_ERR_CUDA.
+ *   - All calls on one device share the one array, and it keeps what the last call
+ *     left in it (each call clears the part that has to start at zero, on `stream`).
+ *     Two calls whose work can overlap on the GPU -- different streams without an
+ *     ordering between them -- race on it and give wrong results: order them.
+ */
+#define DST_STATIC_WORKSPACE_BYTES (4u << 20)
+int dst_densify_static(const void* indices, const void* values, int64_t n_rows, int64_t d, int64_t vocab,
+                       const void* dense_in, void* out, dst_stream_t stream, const dst_opts_t* opts,
+                       void* unique_rows, int32_t* counts, dst_result_t* result);
+
 /* Bytes of device staging memory dst_densify_concat_host needs. */
 size_t dst_host_staging_bytes(int64_t n_rows_total, int64_t d, int64_t vocab, const dst_opts_t* opts);
 

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     dst_densify,
     dst_densify_concat,
     dst_densify_concat_host,
+    dst_densify_static,
     dst_host_staging_bytes,
     dst_kernel_launches,
     dst_profile_events,

@@ -58,6 +58,8 @@ SYMBOLS = {
                                    _vp, _vp, _vp]),
     "dst_densify_concat": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, _vp,
                                           ctypes.POINTER(_Opts), _vp, _sz, _vp, _vp, _vp]),
+    "dst_densify_static": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i64, _vp, _vp, _vp, ctypes.POINTER(_Opts),
+                                          _vp, _vp, _vp]),
     "dst_host_staging_bytes": (_sz, [_i64, _i64, _i64, ctypes.POINTER(_Opts)]),
     "dst_densify_concat_host": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, _vp,
                                                ctypes.POINTER(_Opts), _vp, _sz, _vp, _sz, _vp]),
@@ -229,6 +231,34 @@ def dst_densify(indices: torch.Tensor, values: torch.Tensor, d: int, vocab: int,
                              _ptr(result))
     if rc != 0:
         raise DstError(rc, "dst_densify")
+
+
+STATIC_WORKSPACE_BYTES = 4 << 20   # DST_STATIC_WORKSPACE_BYTES of include/dst.h
+
+
+def dst_densify_static(indices: torch.Tensor, values: torch.Tensor, d: int, vocab: int,
+                       dense_in: Optional[torch.Tensor], out: torch.Tensor,
+                       unique_rows: Optional[torch.Tensor] = None, counts: Optional[torch.Tensor] = None,
+                       result: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Enqueue ``dst_densify_static`` (include/dst.h): ``dst_densify`` for callers that cannot hand
+    over a workspace because they must not allocate device memory where they call from.  The scratch
+    is an array inside the library (``STATIC_WORKSPACE_BYTES`` per GPU), so shapes that need more raise
+    ``DstError`` (workspace too small), and calls that may overlap on the GPU must be ordered by the
+    caller.  Make the first call on a device outside stream capture."""
+    lib = load_library()
+    _check_slice(indices, values, d, out.device)
+    if out.numel() != vocab * d or not out.is_contiguous():
+        raise ValueError("out must be contiguous [vocab, d]")
+    if dense_in is not None and (dense_in.dtype != out.dtype or dense_in.numel() != vocab * d
+                                 or not dense_in.is_contiguous()):
+        raise ValueError("dense_in must be contiguous [vocab, d] in out's dtype")
+    o = _opts(indices.dtype, values.dtype, out.dtype)
+    with torch.cuda.device(out.device):
+        rc = lib.dst_densify_static(_ptr(indices), _ptr(values), indices.shape[0], d, vocab, _ptr(dense_in),
+                                    _ptr(out), _stream_handle(stream), ctypes.byref(o), _ptr(unique_rows),
+                                    _ptr(counts), _ptr(result))
+    if rc != 0:
+        raise DstError(rc, "dst_densify_static")
 
 
 def dst_densify_concat_host(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]], d: int, vocab: int,

@@ -2,6 +2,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
 
 #include "dst_common.cuh"
 
@@ -125,6 +126,35 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     return DST_OK;
 }
 
+// ---- scratch for dst_densify_static ------------------------------------------------
+// Device global memory that belongs to the library itself: every GPU that loads the
+// library holds one copy until the process exits.  In host code this name is only a
+// handle for the runtime's symbol look-up, never a device address; kernels get the
+// address that cudaGetSymbolAddress returns for the current device.
+static __device__ __align__(256) unsigned char g_static_workspace[DST_STATIC_WORKSPACE_BYTES];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mutex;
+static void* g_static_ptr[kMaxDevices];   // device address of the array, per device ordinal
+
+// Address of the array on the current device; looked up once per device.
+static cudaError_t static_workspace(void** ptr) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_workspace);
+        if (e != cudaSuccess) return e;
+        if (!p) return cudaErrorInvalidSymbol;
+        g_static_ptr[dev] = p;
+    }
+    *ptr = g_static_ptr[dev];
+    return cudaSuccess;
+}
+
 }  // namespace dst
 
 using namespace dst;
@@ -172,6 +202,22 @@ int dst_densify_concat(const dst_slice_t* slices, int32_t R, int64_t d, int64_t 
                        size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
     return densify_impl(slices, R, d, vocab, dense_in, out, stream, opts, workspace, workspace_bytes, unique_rows,
                         counts, result);
+}
+
+int dst_densify_static(const void* indices, const void* values, int64_t n_rows, int64_t d, int64_t vocab,
+                       const void* dense_in, void* out, dst_stream_t stream, const dst_opts_t* opts,
+                       void* unique_rows, int32_t* counts, dst_result_t* result) {
+    if (!opts_ok(opts)) return opts ? DST_ERR_UNSUPPORTED : DST_ERR_INVALID_ARG;
+    if (n_rows < 0 || d < 0 || vocab < 0) return DST_ERR_INVALID_ARG;
+    if (n_rows > kMaxRows || vocab > kMaxVocab) return DST_ERR_UNSUPPORTED;
+    if (vocab == 0 || d == 0) return DST_OK;
+    // the shape decides the need; refuse before touching the device
+    if (make_layout(n_rows, 1, d, vocab).total > size_t(DST_STATIC_WORKSPACE_BYTES)) return DST_ERR_WORKSPACE_TOO_SMALL;
+    void* ws = nullptr;
+    if (static_workspace(&ws) != cudaSuccess) return DST_ERR_CUDA;
+    dst_slice_t s{indices, values, n_rows};
+    return densify_impl(&s, 1, d, vocab, dense_in, out, stream, opts, ws, size_t(DST_STATIC_WORKSPACE_BYTES),
+                        unique_rows, counts, result);
 }
 
 size_t dst_host_staging_bytes(int64_t n_rows_total, int64_t d, int64_t vocab, const dst_opts_t* opts) {
