@@ -51,7 +51,7 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     if (vocab == 0 || d == 0) return DST_OK;
     if (!out || !workspace) return DST_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return DST_ERR_INVALID_ARG;
-    const Layout L = make_layout(n_total, R, d, vocab);
+    const Layout L = make_layout(n_total, R, d, vocab, int(dtype_size(opts->value_type)), int(dtype_size(opts->out_type)));
     if (workspace_bytes < L.total) return DST_ERR_WORKSPACE_TOO_SMALL;
 
     char* ws = static_cast<char*>(workspace);
@@ -60,6 +60,7 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     unsigned* digit = reinterpret_cast<unsigned*>(ws + L.off_digit);
     unsigned* desc = reinterpret_cast<unsigned*>(ws + L.off_desc);
     unsigned* nodecnt = reinterpret_cast<unsigned*>(ws + L.off_nodecnt);
+    int2* batches = reinterpret_cast<int2*>(ws + L.off_batches);
     int* offsets = reinterpret_cast<int*>(ws + L.off_offsets);
     unsigned* keys[2] = {reinterpret_cast<unsigned*>(ws + L.off_keys[0]), reinterpret_cast<unsigned*>(ws + L.off_keys[1])};
     unsigned* pos[2] = {reinterpret_cast<unsigned*>(ws + L.off_pos[0]), reinterpret_cast<unsigned*>(ws + L.off_pos[1])};
@@ -69,8 +70,9 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     float* partials = reinterpret_cast<float*>(ws + L.off_partials);
 
     // the fast kernels need 16-byte aligned rows everywhere
-    const int vc = int(16 / dtype_size(opts->value_type));
-    bool vector_ok = d % vc == 0 && aligned16(out) && aligned16(dense_in);
+    const size_t smallest = dtype_size(opts->value_type) < dtype_size(opts->out_type) ? dtype_size(opts->value_type)
+                                                                                      : dtype_size(opts->out_type);
+    bool vector_ok = d % int64_t(16 / smallest) == 0 && aligned16(out) && aligned16(dense_in);
     for (int r = 0; r < R && vector_ok; ++r)
         if (slices[r].n_rows > 0 && !aligned16(slices[r].values)) vector_ok = false;
 
@@ -98,7 +100,7 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     }
     // a3/a5/a6
     if (launch_scan(opts->index_type, hdr, count, offsets, heavy, chunkdesc, unique_rows, counts, result,
-                    int(L.vocab_pad), L.chunk, stream) != cudaSuccess)
+                    batches, int(vocab), int(L.vocab_pad), L.chunk, L.batch_units, stream) != cudaSuccess)
         return DST_ERR_CUDA;
     ++g_launches;
     // a4: least significant digit first; keys/positions ping-pong between two buffers
@@ -115,11 +117,12 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     // a7/a8
     MainArgs a;
     a.hdr = hdr; a.offsets = offsets; a.perm = pos[L.passes & 1]; a.tab = tab; a.heavy = heavy;
-    a.chunkdesc = chunkdesc; a.node_cnt = nodecnt; a.partials = partials; a.dense_in = dense_in; a.out = out;
+    a.chunkdesc = chunkdesc; a.batches = batches; a.node_cnt = nodecnt; a.partials = partials; a.dense_in = dense_in; a.out = out;
     a.result = result; a.d = d; a.vocab = int(vocab); a.n_total = int(n_total); a.R = R; a.chunk = L.chunk;
-    a.chunk_max = int(L.chunk_max);
+    a.chunk_max = int(L.chunk_max); a.upper_max = int(L.upper_max);
+    a.W = a.ncb = a.slot_bytes = a.n_slots = 0;   // set by the launcher
     if (t_ev_before && cudaEventRecord(t_ev_before, stream) != cudaSuccess) return DST_ERR_CUDA;
-    if (launch_reduce_rows(a, opts->value_type, opts->out_type, vector_ok, sm_count() * 4, stream) != cudaSuccess)
+    if (launch_reduce_rows(a, opts->value_type, opts->out_type, vector_ok, sm_count(), stream) != cudaSuccess)
         return DST_ERR_CUDA;
     ++g_launches;
     if (t_ev_after && cudaEventRecord(t_ev_after, stream) != cudaSuccess) return DST_ERR_CUDA;
@@ -186,7 +189,7 @@ const char* dst_status_string(int status) {
 size_t dst_workspace_bytes(int64_t n_rows_total, int32_t R, int64_t d, int64_t vocab, const dst_opts_t* opts) {
     if (!opts_ok(opts) || n_rows_total < 0 || n_rows_total > kMaxRows || R < 0 || d < 0 || vocab < 0 || vocab > kMaxVocab)
         return 0;
-    return make_layout(n_rows_total, R, d, vocab).total;
+    return make_layout(n_rows_total, R, d, vocab, int(dtype_size(opts->value_type)), int(dtype_size(opts->out_type))).total;
 }
 
 int dst_densify(const void* indices, const void* values, int64_t n_rows, int64_t d, int64_t vocab,
@@ -212,7 +215,8 @@ int dst_densify_static(const void* indices, const void* values, int64_t n_rows, 
     if (n_rows > kMaxRows || vocab > kMaxVocab) return DST_ERR_UNSUPPORTED;
     if (vocab == 0 || d == 0) return DST_OK;
     // the shape decides the need; refuse before touching the device
-    if (make_layout(n_rows, 1, d, vocab).total > size_t(DST_STATIC_WORKSPACE_BYTES)) return DST_ERR_WORKSPACE_TOO_SMALL;
+    if (make_layout(n_rows, 1, d, vocab, int(dtype_size(opts->value_type)), int(dtype_size(opts->out_type))).total >
+        size_t(DST_STATIC_WORKSPACE_BYTES)) return DST_ERR_WORKSPACE_TOO_SMALL;
     void* ws = nullptr;
     if (static_workspace(&ws) != cudaSuccess) return DST_ERR_CUDA;
     dst_slice_t s{indices, values, n_rows};

@@ -16,8 +16,16 @@ constexpr int kTile = kSortThreads * kSortItems;  // 2048 keys per CTA
 constexpr int kHashSlots = 4096;            // per-CTA key aggregation table (> kTile distinct keys never happen)
 constexpr int kMaxPasses = 4;               // 8-bit digits, keys below 2^31
 constexpr int kFanIn = 16;                  // children per node of the heavy-row combine tree
-constexpr int kRowsPerBatch = 4;            // output rows per light work item
-constexpr int kMainThreads = 256;
+constexpr int kMaxBatchUnits = 31;          // a light work item holds rows worth at most this many units (+ one row)
+constexpr int kMaxChunk = 64;               // entries per chunk of a heavy row (at most)
+constexpr int kPipeWarpsTotal = 148 * 8;    // warps the row-reduction kernel runs with on a B200 (sizes the work items)
+constexpr int kPipeWarps = 4;               // row-reduction kernel: warps per CTA, each with its own slot ring
+constexpr int kPipeThreads = kPipeWarps * 32;
+constexpr int kPipeSlots = 6;               // ring slots per warp
+constexpr int kPipeHeaderReserve = 1024;    // mbarriers in front of the slots
+constexpr int kMaxBlockCols = 1024;         // columns per column block (32 fp32 accumulators per lane)
+constexpr int kSmemPerSm = 227 * 1024;
+constexpr long long kWaitCycles = 1LL << 31; // SM clock cycles (about a second) before an mbarrier wait gives up
 constexpr int kScanThreads = 1024;
 constexpr int kScanItems = 16;              // counters per thread and round in the scan kernel
 constexpr int kSmCount = 148;               // B200; only used to pick the chunk length
@@ -37,11 +45,12 @@ struct WsHeader {          // zeroed at the start of every call
     int n_chunks;          // work items those rows are split into
     int n_upper;           // combine-tree nodes above the chunk level
     int max_segment;
-    int pad0;
+    unsigned int done;     // CTAs of the row-reduction kernel that have finished
     unsigned long long n_bad;
     unsigned int ticket[kMaxPasses];
     unsigned int work_counter;
-    unsigned int pad1[3];
+    int n_batches;         // light work items (row batches)
+    unsigned int pad1[2];
 };
 static_assert(sizeof(WsHeader) == 72, "header layout");
 
@@ -75,9 +84,9 @@ struct ChunkDesc {         // one chunk work item
 
 struct Layout {
     int64_t n_rows, vocab, d;
-    int R, chunk, passes;
-    int64_t n_tiles, vocab_pad, heavy_max, chunk_max, upper_max;
-    size_t off_header, off_count, off_digit, off_desc, off_nodecnt, zero_bytes;
+    int R, chunk, passes, batch_units;
+    int64_t n_tiles, vocab_pad, heavy_max, chunk_max, upper_max, batch_max;
+    size_t off_header, off_count, off_digit, off_desc, off_nodecnt, off_batches, zero_bytes;
     size_t off_offsets, off_keys[2], off_pos[2], off_tab, off_heavy, off_chunkdesc, off_partials;
     size_t total;
 };
@@ -90,6 +99,7 @@ struct MainArgs {
     const SliceEntry* tab;
     const HeavyInfo* heavy;
     const ChunkDesc* chunkdesc;
+    const int2* batches;   // per row batch: first row + 1 (0: empty batch), last row + 1
     unsigned* node_cnt;
     float* partials;
     const void* dense_in;
@@ -101,20 +111,46 @@ struct MainArgs {
     int R;
     int chunk;
     int chunk_max;   // partial rows of the chunk level; upper nodes follow
+    int upper_max;   // combine-tree arrival counters per column block
+    int W;           // columns per column block
+    int ncb;         // column blocks per row
+    int slot_bytes;
+    int n_slots;
 };
+
+// How the row-reduction kernel cuts rows into column blocks and shared memory into slots.
+struct PipeShape { int K, W, ncb, slot_bytes, n_slots, ctas_per_sm; };
+inline PipeShape pipe_shape(int value_size, int out_size, int64_t d) {
+    PipeShape p{};
+    const int vc = 16 / value_size;                        // columns per 16-byte group of a value row
+    const int64_t w = d < kMaxBlockCols ? d : kMaxBlockCols;
+    p.W = int(w > 0 ? w : 1);
+    p.ncb = int(d > 0 ? (d + p.W - 1) / p.W : 1);
+    p.K = 1;
+    while (p.K * 32 * vc < p.W) p.K *= 2;                  // 16-byte groups per lane
+    const int widest = value_size > out_size ? value_size : out_size;
+    p.slot_bytes = (p.W * widest + 127) / 128 * 128;
+    p.n_slots = kPipeSlots;
+    const int per_cta = kPipeHeaderReserve + kPipeWarps * p.n_slots * p.slot_bytes + 1024;   // + the driver's reserve
+    int c = kSmemPerSm / per_cta;
+    p.ctas_per_sm = c < 1 ? 1 : (c > 8 ? 8 : c);
+    return p;
+}
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Everything about the workspace follows from the shapes alone, so the same
 // shapes always give the same chunking and therefore the same summation order.
-inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab) {
+inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab, int value_size, int out_size) {
     Layout L{};
     L.n_rows = n_rows; L.vocab = vocab; L.d = d; L.R = R;
-    // chunk length: keep work items near 1/32 of an SM's fair share of rows
-    int64_t units = 2 * vocab + n_rows;
-    int64_t per = units / (int64_t(kSmCount) * 32);
+    // Work-item sizes: about a third of a warp's fair share of units (one unit = one source row),
+    // so that the tail of the row-reduction kernel stays short.
+    const int64_t share = (vocab + n_rows) / (int64_t(kPipeWarpsTotal) * 3);
     int c = 16;
-    while (c < 256 && c * 2 <= per) c *= 2;
+    while (c < kMaxChunk && c * 2 <= share) c *= 2;
+    L.batch_units = int(share < 8 ? 8 : (share > kMaxBatchUnits ? kMaxBatchUnits : share));
+    L.batch_max = (vocab + n_rows) / L.batch_units + 2;
     L.chunk = c;
     int bits = 0;
     while (bits < 31 && (int64_t(1) << bits) < vocab) ++bits;   // keys are < vocab <= 2^bits
@@ -130,7 +166,8 @@ inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab) {
     L.off_count = take(size_t(L.vocab_pad) * 4);
     L.off_digit = take(size_t(kMaxPasses) * 256 * 4);
     L.off_desc = take(size_t(L.passes) * size_t(L.n_tiles) * 256 * 4);
-    L.off_nodecnt = take(size_t(L.upper_max) * 4);
+    L.off_nodecnt = take(size_t(L.upper_max) * size_t(pipe_shape(value_size, out_size, d).ncb) * 4);
+    L.off_batches = take(size_t(L.batch_max) * 8);
     L.zero_bytes = o;
     L.off_offsets = take(size_t(L.vocab_pad + kScanItems) * 4);
     L.off_keys[0] = take(size_t(n_rows) * 4);
@@ -151,11 +188,11 @@ cudaError_t launch_hist(const HistParams& P, int grid_x, int index_type, WsHeade
                         cudaStream_t stream);
 cudaError_t launch_scan(int index_type, WsHeader* hdr, const unsigned* count, int* offsets, HeavyInfo* heavy,
                         ChunkDesc* chunkdesc, void* unique_rows, int* counts_out, dst_result_t* result,
-                        int vocab_pad, int chunk, cudaStream_t stream);
+                        int2* batches, int vocab, int vocab_pad, int chunk, int batch_units, cudaStream_t stream);
 cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
                               unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
                               int pass, int capacity, cudaStream_t stream);
-cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int grid,
+cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,
                                cudaStream_t stream);
 
 // ---- device helpers ---------------------------------------------------------

@@ -71,39 +71,39 @@ k_hist(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, unsigne
 // ---------------------------------------------------------------------------
 // a3 + a5 + a6: exclusive scan of the histogram, unique compaction, heavy-row chunking
 // ---------------------------------------------------------------------------
-struct Scan5 { int v[5]; };   // 0 offset, 1 unique, 2 heavy rows, 3 chunks, 4 upper nodes
+struct Scan5 { int v[6]; };   // 0 offset, 1 unique, 2 heavy rows, 3 chunks, 4 upper nodes, 5 units of the light work items
 
-__device__ __forceinline__ Scan5 block_exclusive_scan(Scan5 x, Scan5& total, int (*sm)[5]) {
+__device__ __forceinline__ Scan5 block_exclusive_scan(Scan5 x, Scan5& total, int (*sm)[6]) {
     const int lane = lane_id(), warp = warp_id();
     Scan5 inc = x;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
 #pragma unroll
-        for (int q = 0; q < 5; ++q) {
+        for (int q = 0; q < 6; ++q) {
             int t = __shfl_up_sync(0xFFFFFFFFu, inc.v[q], o);
             if (lane >= o) inc.v[q] += t;
         }
     }
     if (lane == 31) {
 #pragma unroll
-        for (int q = 0; q < 5; ++q) sm[warp][q] = inc.v[q];
+        for (int q = 0; q < 6; ++q) sm[warp][q] = inc.v[q];
     }
     __syncthreads();
     if (warp == 0) {
         Scan5 w;
 #pragma unroll
-        for (int q = 0; q < 5; ++q) w.v[q] = sm[lane][q];
+        for (int q = 0; q < 6; ++q) w.v[q] = sm[lane][q];
         Scan5 winc = w;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
 #pragma unroll
-            for (int q = 0; q < 5; ++q) {
+            for (int q = 0; q < 6; ++q) {
                 int t = __shfl_up_sync(0xFFFFFFFFu, winc.v[q], o);
                 if (lane >= o) winc.v[q] += t;
             }
         }
 #pragma unroll
-        for (int q = 0; q < 5; ++q) {
+        for (int q = 0; q < 6; ++q) {
             sm[lane][q] = winc.v[q] - w.v[q];          // exclusive prefix of this warp
             if (lane == 31) sm[32][q] = winc.v[q];     // block total
         }
@@ -111,7 +111,7 @@ __device__ __forceinline__ Scan5 block_exclusive_scan(Scan5 x, Scan5& total, int
     __syncthreads();
     Scan5 ex;
 #pragma unroll
-    for (int q = 0; q < 5; ++q) {
+    for (int q = 0; q < 6; ++q) {
         ex.v[q] = inc.v[q] - x.v[q] + sm[warp][q];
         total.v[q] = sm[32][q];
     }
@@ -123,8 +123,9 @@ template <typename IT>
 __global__ void __launch_bounds__(kScanThreads)
 k_scan(WsHeader* __restrict__ hdr, const unsigned* __restrict__ count, int* __restrict__ offsets,
        HeavyInfo* __restrict__ heavy, ChunkDesc* __restrict__ chunkdesc, IT* __restrict__ unique_rows,
-       int* __restrict__ counts_out, dst_result_t* __restrict__ result, int vocab_pad, int chunk) {
-    __shared__ int sm[33][5];
+       int* __restrict__ counts_out, dst_result_t* __restrict__ result, int2* __restrict__ batches, int vocab,
+       int vocab_pad, int chunk, int batch_units) {
+    __shared__ int sm[33][6];
     __shared__ int smax[32];
     Scan5 carry{};
     int maxseg = 0;
@@ -149,6 +150,7 @@ k_scan(WsHeader* __restrict__ hdr, const unsigned* __restrict__ count, int* __re
             int cc = (int)c[q];
             mine.v[0] += cc;
             mine.v[1] += cc > 0;
+            if (e0 + q < vocab) mine.v[5] += cc > chunk ? 1 : cc + 1;
             if (cc > chunk) {
                 int n = (cc + chunk - 1) / chunk;
                 mine.v[2] += 1; mine.v[3] += n; mine.v[4] += upper_nodes(n);
@@ -158,8 +160,11 @@ k_scan(WsHeader* __restrict__ hdr, const unsigned* __restrict__ count, int* __re
         Scan5 total;
         Scan5 run = block_exclusive_scan(mine, total, sm);
 #pragma unroll
-        for (int q = 0; q < 5; ++q) run.v[q] += carry.v[q];
+        for (int q = 0; q < 6; ++q) run.v[q] += carry.v[q];
         if (e0 < vocab_pad) {
+            // units of the row before this thread's first one (decides whether that row opens a batch)
+            int prev_cost = 0;
+            if (e0 > 0) { int pc = (int)count[e0 - 1]; prev_cost = pc > chunk ? 1 : pc + 1; }
             int o[kScanItems];
 #pragma unroll
             for (int q = 0; q < kScanItems; ++q) {
@@ -176,13 +181,23 @@ k_scan(WsHeader* __restrict__ hdr, const unsigned* __restrict__ count, int* __re
                     run.v[2] += 1; run.v[3] += n; run.v[4] += upper_nodes(n);
                 }
                 run.v[0] += cc;
+                if (e0 + q < vocab) {
+                    // light work items: row v belongs to batch floor(units before v / batch_units)
+                    const int cost = cc > chunk ? 1 : cc + 1;
+                    const int b = run.v[5] / batch_units;
+                    const int v = e0 + q;
+                    if (v == 0 || (run.v[5] - prev_cost) / batch_units != b) batches[b].x = v + 1;
+                    if (v == vocab - 1 || (run.v[5] + cost) / batch_units != b) batches[b].y = v + 1;
+                    run.v[5] += cost;
+                    prev_cost = cost;
+                }
             }
             int4* dst = reinterpret_cast<int4*>(offsets + e0);
 #pragma unroll
             for (int q = 0; q < kScanItems / 4; ++q) dst[q] = make_int4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
         }
 #pragma unroll
-        for (int q = 0; q < 5; ++q) carry.v[q] += total.v[q];
+        for (int q = 0; q < 6; ++q) carry.v[q] += total.v[q];
     }
     for (int o = 16; o > 0; o >>= 1) maxseg = max(maxseg, __shfl_down_sync(0xFFFFFFFFu, maxseg, o));
     if (lane_id() == 0) smax[warp_id()] = maxseg;
@@ -196,6 +211,7 @@ k_scan(WsHeader* __restrict__ hdr, const unsigned* __restrict__ count, int* __re
         hdr->n_chunks = carry.v[3];
         hdr->n_upper = carry.v[4];
         hdr->max_segment = maxseg;
+        hdr->n_batches = carry.v[5] > 0 ? (carry.v[5] - 1) / batch_units + 1 : 0;
         unsigned long long bad = hdr->n_bad;
         if (bad) raise_status(hdr, DST_ERR_INDEX_OUT_OF_RANGE);
         if (result) {
@@ -336,15 +352,15 @@ cudaError_t launch_hist(const HistParams& P, int grid_x, int index_type, WsHeade
 
 cudaError_t launch_scan(int index_type, WsHeader* hdr, const unsigned* count, int* offsets, HeavyInfo* heavy,
                         ChunkDesc* chunkdesc, void* unique_rows, int* counts_out, dst_result_t* result,
-                        int vocab_pad, int chunk, cudaStream_t stream) {
+                        int2* batches, int vocab, int vocab_pad, int chunk, int batch_units, cudaStream_t stream) {
     if (index_type == DST_I64)
         k_scan<long long><<<1, kScanThreads, 0, stream>>>(hdr, count, offsets, heavy, chunkdesc,
                                                           static_cast<long long*>(unique_rows), counts_out, result,
-                                                          vocab_pad, chunk);
+                                                          batches, vocab, vocab_pad, chunk, batch_units);
     else
         k_scan<int><<<1, kScanThreads, 0, stream>>>(hdr, count, offsets, heavy, chunkdesc,
-                                                    static_cast<int*>(unique_rows), counts_out, result, vocab_pad,
-                                                    chunk);
+                                                    static_cast<int*>(unique_rows), counts_out, result, batches,
+                                                    vocab, vocab_pad, chunk, batch_units);
     return cudaGetLastError();
 }
 

@@ -7,13 +7,22 @@
 // the operation.  It is HBM-bound: every value row, every dense_in row and every
 // out row crosses the memory bus exactly once; no tensor cores are involved.
 //
-// Work decomposition (one warp per work item, items handed out by a counter):
+// Structure: persistent CTAs of kPipeWarps independent warps.  Each warp owns a small ring
+// of shared-memory slots and streams "units" (one source row of one column block each)
+// through it: lane 0 issues one bulk asynchronous copy (cp.async.bulk, completion on an
+// mbarrier) per unit, up to n_slots ahead of the unit the warp is adding into its fp32
+// registers, so the bytes in flight are set by shared memory, not by registers.  The
+// units of a work item are laid out flat across the lanes (value rows of a segment, then
+// the unit that closes the output row with its dense_in row), so the copies of one
+// output row overlap with those of its neighbours.  The warp that read a slot is the
+// one that refills it, so only "full" barriers are needed.
+// Work items:
 //   chunk items   `chunk` consecutive entries of a heavy row's segment -> fp32 partial row;
 //                 partials are combined by a fixed fan-in tree whose nodes are
-//                 evaluated by whichever warp arrives last (children always summed
+//                 evaluated by whichever CTA arrives last (children always summed
 //                 in index order, so the result does not depend on timing)
-//   row batches   kRowsPerBatch consecutive output rows that are not heavy
-// A lane owns VC consecutive columns per 16-byte value load and K such groups.
+//   row batches   consecutive output rows that are not heavy, about batch_units units' worth
+// Rows wider than one slot are processed as independent column blocks.
 #include "dst_common.cuh"
 
 namespace dst {
@@ -25,6 +34,10 @@ template <int VC> __device__ __forceinline__ void zero(Acc<VC>& a) {
 #pragma unroll
     for (int i = 0; i < VC; ++i) a.x[i] = 0.f;
 }
+template <int VC> __device__ __forceinline__ void add(Acc<VC>& a, const Acc<VC>& b) {
+#pragma unroll
+    for (int i = 0; i < VC; ++i) a.x[i] += b.x[i];
+}
 
 __device__ __forceinline__ void unpack_bf16x2(unsigned w, float& lo, float& hi) {
     lo = __uint_as_float(w << 16);
@@ -35,43 +48,23 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<unsigned*>(&t);
 }
 
-// read-only input rows (never written during the kernel)
-__device__ __forceinline__ void load_in(const float* p, Acc<4>& a) {
-    float4 t = __ldg(reinterpret_cast<const float4*>(p));
-    a.x[0] = t.x; a.x[1] = t.y; a.x[2] = t.z; a.x[3] = t.w;
-}
-__device__ __forceinline__ void load_in(const float* p, Acc<8>& a) {
-    float4 t = __ldg(reinterpret_cast<const float4*>(p));
-    float4 u = __ldg(reinterpret_cast<const float4*>(p) + 1);
-    a.x[0] = t.x; a.x[1] = t.y; a.x[2] = t.z; a.x[3] = t.w;
-    a.x[4] = u.x; a.x[5] = u.y; a.x[6] = u.z; a.x[7] = u.w;
-}
-__device__ __forceinline__ void load_in(const __nv_bfloat16* p, Acc<8>& a) {
-    uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
-    unpack_bf16x2(t.x, a.x[0], a.x[1]); unpack_bf16x2(t.y, a.x[2], a.x[3]);
-    unpack_bf16x2(t.z, a.x[4], a.x[5]); unpack_bf16x2(t.w, a.x[6], a.x[7]);
-}
-__device__ __forceinline__ void load_in(const __nv_bfloat16* p, Acc<4>& a) {
-    uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
-    unpack_bf16x2(t.x, a.x[0], a.x[1]); unpack_bf16x2(t.y, a.x[2], a.x[3]);
-}
-// dense_in may alias out: plain (coherent) loads
-__device__ __forceinline__ void load_dense(const float* p, Acc<4>& a) {
+// VC consecutive elements at p (shared or global memory, generic address) -> fp32
+__device__ __forceinline__ void load_elems(const float* p, Acc<4>& a) {
     float4 t = *reinterpret_cast<const float4*>(p);
     a.x[0] = t.x; a.x[1] = t.y; a.x[2] = t.z; a.x[3] = t.w;
 }
-__device__ __forceinline__ void load_dense(const float* p, Acc<8>& a) {
+__device__ __forceinline__ void load_elems(const float* p, Acc<8>& a) {
     float4 t = *reinterpret_cast<const float4*>(p);
     float4 u = *(reinterpret_cast<const float4*>(p) + 1);
     a.x[0] = t.x; a.x[1] = t.y; a.x[2] = t.z; a.x[3] = t.w;
     a.x[4] = u.x; a.x[5] = u.y; a.x[6] = u.z; a.x[7] = u.w;
 }
-__device__ __forceinline__ void load_dense(const __nv_bfloat16* p, Acc<8>& a) {
+__device__ __forceinline__ void load_elems(const __nv_bfloat16* p, Acc<8>& a) {
     uint4 t = *reinterpret_cast<const uint4*>(p);
     unpack_bf16x2(t.x, a.x[0], a.x[1]); unpack_bf16x2(t.y, a.x[2], a.x[3]);
     unpack_bf16x2(t.z, a.x[4], a.x[5]); unpack_bf16x2(t.w, a.x[6], a.x[7]);
 }
-__device__ __forceinline__ void load_dense(const __nv_bfloat16* p, Acc<4>& a) {
+__device__ __forceinline__ void load_elems(const __nv_bfloat16* p, Acc<4>& a) {
     uint2 t = *reinterpret_cast<const uint2*>(p);
     unpack_bf16x2(t.x, a.x[0], a.x[1]); unpack_bf16x2(t.y, a.x[2], a.x[3]);
 }
@@ -90,7 +83,7 @@ __device__ __forceinline__ void store_out(__nv_bfloat16* p, const Acc<8>& a) {
 __device__ __forceinline__ void store_out(__nv_bfloat16* p, const Acc<4>& a) {
     __stcs(reinterpret_cast<uint2*>(p), make_uint2(pack_bf16x2(a.x[0], a.x[1]), pack_bf16x2(a.x[2], a.x[3])));
 }
-// partial rows: written by one warp, read by another through L2
+// partial rows: written by one CTA, read by another through L2
 template <int VC> __device__ __forceinline__ void store_partial(float* p, const Acc<VC>& a) {
 #pragma unroll
     for (int i = 0; i < VC; i += 4)
@@ -102,16 +95,6 @@ template <int VC> __device__ __forceinline__ void load_partial(const float* p, A
         float4 t = __ldcg(reinterpret_cast<const float4*>(p + i));
         a.x[i] = t.x; a.x[i + 1] = t.y; a.x[i + 2] = t.z; a.x[i + 3] = t.w;
     }
-}
-template <int VC> __device__ __forceinline__ void add(Acc<VC>& a, const Acc<VC>& b) {
-#pragma unroll
-    for (int i = 0; i < VC; ++i) a.x[i] += b.x[i];
-}
-
-template <typename T> __device__ __forceinline__ const T* shfl_ptr(const T* p, int src) {
-    unsigned long long u = reinterpret_cast<unsigned long long>(p);
-    u = __shfl_sync(0xFFFFFFFFu, u, src);
-    return reinterpret_cast<const T*>(u);
 }
 
 // position in the virtual concatenation -> address of that value row
@@ -131,113 +114,109 @@ __device__ __forceinline__ const VT* resolve_row(const MainArgs& a, unsigned p) 
     return base + local * a.d;
 }
 
+// ---- mbarrier / bulk-copy primitives (shared::cta addresses) -----------------------
+__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up when the limit is reached or another thread has given up.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long start = clock64();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag || clock64() - start > kWaitCycles) return false;
+    }
+}
+// global -> this CTA's shared memory, 16-byte aligned on both sides, bytes % 16 == 0
+__device__ __forceinline__ void bulk_load(unsigned dst_smem, const void* src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// ---- per-warp slot ring --------------------------------------------------------------
+enum : int {
+    kUnitAdd = 1,        // slot holds a value row: add it
+    kUnitFinal = 2,      // finish output row y (slot holds its dense_in row unless there is no dense_in)
+    kUnitCopy = 4,       // with kUnitFinal: nobody names the row, out = dense_in bit for bit
+    kUnitChunkEnd = 8    // last entry of chunk y: store the partial row, climb the tree
+};
+
+// A block of at most 32 units, one per lane.
+struct UnitBlock {
+    const void* src;     // first byte to copy (nullptr: nothing to copy)
+    unsigned bytes;
+    int kind;
+    int y;               // output row (kUnitFinal) or chunk id (kUnitChunkEnd)
+};
+
 template <typename VT, typename OT, int K>
-struct RowReducer {
-    static constexpr int VC = 16 / sizeof(VT);          // columns per 16-byte value load
-    static constexpr int kColsPerPass = K * 32 * VC;
+struct WarpPipe {
+    static constexpr int VC = 16 / sizeof(VT);     // columns per 16-byte group of a value row
     const MainArgs& a;
     const int lane;
-    __device__ RowReducer(const MainArgs& args) : a(args), lane(lane_id()) {}
+    const unsigned ring;      // shared address of this warp's first slot
+    const unsigned bars;      // shared address of this warp's first mbarrier (one per slot)
+    char* const ring_ptr;     // generic address of the first slot
+    volatile int* const abort_flag;
+    int islot;                // slot the next issued unit goes to
+    int cslot;                // slot of the next unit to consume
+    unsigned cphase;          // bit s: parity to wait for on slot s
+    unsigned issued_mask;     // slots with a copy that may still be in flight
 
-    __device__ __forceinline__ long long col(int cb, int k) const { return (long long)cb + (long long)(k * 32 + lane) * VC; }
+    __device__ WarpPipe(const MainArgs& args, unsigned ring_addr, unsigned bar_addr, char* ring_generic, volatile int* ab)
+        : a(args), lane(lane_id()), ring(ring_addr), bars(bar_addr), ring_ptr(ring_generic), abort_flag(ab), islot(0),
+          cslot(0), cphase(0u), issued_mask(0u) {}
 
-    // acc += sum of value rows perm[begin .. begin+len), ascending
-    __device__ __forceinline__ void accumulate_segment(Acc<VC> (&acc)[K], int begin, int len, long long cb) const {
-        for (int base = 0; base < len; base += 32) {
-            const int m = min(32, len - base);
-            const VT* ptr = nullptr;
-            if (lane < m) {
-                unsigned p = a.perm[begin + base + lane];
-                if (p < (unsigned)a.n_total) ptr = resolve_row<VT>(a, p);
-            }
-            for (int j = 0; j < m; j += 2) {
-                const VT* pa = shfl_ptr(ptr, j);
-                const VT* pb = shfl_ptr(ptr, (j + 1) & 31);
-                if (j + 1 >= m) pb = nullptr;
-                Acc<VC> va[K], vb[K];
-#pragma unroll
-                for (int k = 0; k < K; ++k) {
-                    long long c = col(cb, k);
-                    zero(va[k]); zero(vb[k]);
-                    if (c < a.d) {
-                        if (pa) load_in(pa + c, va[k]);
-                        if (pb) load_in(pb + c, vb[k]);
-                    }
-                }
-#pragma unroll
-                for (int k = 0; k < K; ++k) { add(acc[k], va[k]); add(acc[k], vb[k]); }
+    __device__ __forceinline__ int col(int k) const { return (k * 32 + lane) * VC; }
+
+    // unit j of the block goes into the next slot (lane 0 talks to the copy engine)
+    __device__ __forceinline__ void issue(const UnitBlock& b, int j) {
+        const unsigned long long s = __shfl_sync(0xFFFFFFFFu, reinterpret_cast<unsigned long long>(b.src), j);
+        const unsigned bytes = __shfl_sync(0xFFFFFFFFu, b.bytes, j);
+        if (lane == 0) {
+            const unsigned bar = bars + 8u * (unsigned)islot;
+            if (bytes) {
+                mbar_arrive_expect_tx(bar, bytes);
+                bulk_load(ring + (unsigned)islot * (unsigned)a.slot_bytes, reinterpret_cast<const void*>(s), bytes, bar);
+            } else {
+                mbar_arrive(bar);
             }
         }
-    }
-
-    __device__ __forceinline__ void finish_row(Acc<VC> (&acc)[K], int row, long long cb) const {
-        const OT* din = static_cast<const OT*>(a.dense_in);
-        OT* out = static_cast<OT*>(a.out);
-#pragma unroll
-        for (int k = 0; k < K; ++k) {
-            long long c = col(cb, k);
-            if (c < a.d) {
-                if (din) { Acc<VC> dn; load_dense(din + (long long)row * a.d + c, dn); add(acc[k], dn); }
-                store_out(out + (long long)row * a.d + c, acc[k]);
-            }
-        }
-    }
-
-    // rows nobody names: a straight copy of dense_in (bit-exact), or zeros
-    __device__ __forceinline__ void copy_row(int row) const {
-        const OT* din = static_cast<const OT*>(a.dense_in);
-        OT* out = static_cast<OT*>(a.out);
-        for (long long cb = 0; cb < a.d; cb += kColsPerPass) {
-            Acc<VC> t[K];
-#pragma unroll
-            for (int k = 0; k < K; ++k) {
-                long long c = col(cb, k);
-                zero(t[k]);
-                if (din && c < a.d) load_dense(din + (long long)row * a.d + c, t[k]);
-            }
-#pragma unroll
-            for (int k = 0; k < K; ++k) {
-                long long c = col(cb, k);
-                if (c < a.d) store_out(out + (long long)row * a.d + c, t[k]);
-            }
-        }
-    }
-
-    __device__ void do_row_batch(int batch) const {
-        const int v0 = batch * kRowsPerBatch;
-        const int nrows = min(kRowsPerBatch, a.vocab - v0);
-        int o = 0;
-        if (lane <= nrows) o = a.offsets[v0 + lane];
-        for (int i = 0; i < nrows; ++i) {
-            const int beg = __shfl_sync(0xFFFFFFFFu, o, i);
-            const int cnt = __shfl_sync(0xFFFFFFFFu, o, i + 1) - beg;
-            if (cnt > a.chunk) continue;                 // heavy: produced by the chunk items
-            if (cnt == 0) { copy_row(v0 + i); continue; }
-            for (long long cb = 0; cb < a.d; cb += kColsPerPass) {
-                Acc<VC> acc[K];
-#pragma unroll
-                for (int k = 0; k < K; ++k) zero(acc[k]);
-                accumulate_segment(acc, beg, cnt, cb);
-                finish_row(acc, v0 + i, cb);
-            }
-        }
+        issued_mask |= 1u << islot;
+        islot = islot + 1 == a.n_slots ? 0 : islot + 1;
     }
 
     __device__ __forceinline__ float* partial_row(int slot) const { return a.partials + (long long)slot * a.d; }
 
     // acc = child[0] + child[1] + ... in index order
-    __device__ __forceinline__ void sum_children(Acc<VC> (&acc)[K], int first_slot, int n, long long cb) const {
+    __device__ __forceinline__ void sum_children(Acc<VC> (&acc)[K], int first_slot, int n, long long cb, int wcols) const {
 #pragma unroll
         for (int k = 0; k < K; ++k) zero(acc[k]);
         for (int c = 0; c < n; c += 2) {
-            const float* pa = partial_row(first_slot + c);
-            const float* pb = (c + 1 < n) ? partial_row(first_slot + c + 1) : nullptr;
+            const float* pa = partial_row(first_slot + c) + cb;
+            const float* pb = (c + 1 < n) ? partial_row(first_slot + c + 1) + cb : nullptr;
             Acc<VC> va[K], vb[K];
 #pragma unroll
             for (int k = 0; k < K; ++k) {
-                long long cc = col(cb, k);
+                const int cc = col(k);
                 zero(va[k]); zero(vb[k]);
-                if (cc < a.d) {
+                if (cc < wcols) {
                     load_partial(pa + cc, va[k]);
                     if (pb) load_partial(pb + cc, vb[k]);
                 }
@@ -247,22 +226,22 @@ struct RowReducer {
         }
     }
 
-    __device__ void do_chunk(int cid) const {
-        const ChunkDesc cd = a.chunkdesc[cid];
-        for (long long cb = 0; cb < a.d; cb += kColsPerPass) {
-            Acc<VC> acc[K];
-#pragma unroll
-            for (int k = 0; k < K; ++k) zero(acc[k]);
-            accumulate_segment(acc, cd.begin, cd.len, cb);
-            float* pr = partial_row(cid);
+    // The chunk's sum is in acc: store it as a partial row and climb the combine tree while this
+    // warp is the last child to arrive.
+    __device__ void finish_chunk(Acc<VC> (&acc)[K], int cid, int cblk) const {
+        const long long cb = (long long)cblk * a.W;
+        const int wcols = (int)min((long long)a.W, a.d - cb);
+        {
+            float* pr = partial_row(cid) + cb;
 #pragma unroll
             for (int k = 0; k < K; ++k) {
-                long long c = col(cb, k);
-                if (c < a.d) store_partial(pr + c, acc[k]);
+                const int c = col(k);
+                if (c < wcols) store_partial(pr + c, acc[k]);
             }
         }
-        // climb the combine tree while this warp is the last child to arrive
+        const ChunkDesc cd = a.chunkdesc[cid];
         const HeavyInfo hi = a.heavy[cd.heavy];
+        unsigned* node_cnt = a.node_cnt + (size_t)cblk * (size_t)a.upper_max;
         int j = cid - hi.chunk_base;     // index inside the current level
         int n_level = hi.n_chunks;       // nodes on the current level
         int child_first = hi.chunk_base; // partial slot of node 0 of the current level
@@ -275,49 +254,226 @@ struct RowReducer {
             __threadfence();
             __syncwarp();
             int last = 0;
-            if (lane == 0) last = atomicAdd(&a.node_cnt[node], 1u) == (unsigned)(n_children - 1);
+            if (lane == 0) last = atomicAdd(&node_cnt[node], 1u) == (unsigned)(n_children - 1);
             last = __shfl_sync(0xFFFFFFFFu, last, 0);
             if (!last) return;
             __threadfence();
-            const int first_child_slot = child_first + parent * kFanIn;
             const bool root = n_parent == 1;
-            for (long long cb = 0; cb < a.d; cb += kColsPerPass) {
-                Acc<VC> acc[K];
-                sum_children(acc, first_child_slot, n_children, cb);
-                if (root) {
-                    finish_row(acc, hi.row, cb);
-                } else {
-                    float* pr = partial_row(a.chunk_max + node);
+            sum_children(acc, child_first + parent * kFanIn, n_children, cb, wcols);
+            if (root) {
+                const OT* din = static_cast<const OT*>(a.dense_in);
+                OT* out = static_cast<OT*>(a.out) + (long long)hi.row * a.d + cb;
 #pragma unroll
-                    for (int k = 0; k < K; ++k) {
-                        long long c = col(cb, k);
-                        if (c < a.d) store_partial(pr + c, acc[k]);
+                for (int k = 0; k < K; ++k) {
+                    const int c = col(k);
+                    if (c < wcols) {
+                        if (din) { Acc<VC> dn; load_elems(din + (long long)hi.row * a.d + cb + c, dn); add(acc[k], dn); }
+                        store_out(out + c, acc[k]);
                     }
                 }
+                return;
             }
-            if (root) return;
+            float* pr = partial_row(a.chunk_max + node) + cb;
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                const int c = col(k);
+                if (c < wcols) store_partial(pr + c, acc[k]);
+            }
             child_first = a.chunk_max + hi.upper_base + upper_off;
             upper_off += n_parent;
             j = parent;
             n_level = n_parent;
         }
     }
+
+    __device__ __forceinline__ void give_up() const {
+        raise_status(a.hdr, DST_ERR_TIMEOUT);
+        *abort_flag = 1;
+    }
+
+    // Stream the n units of a block (lane j holds unit j) through the ring: up to n_slots copies in
+    // flight, consumed in order.  Returns false when a wait gave up.
+    __device__ bool run_block(Acc<VC> (&acc)[K], const UnitBlock& b, int n, int cblk) {
+        const long long cb = (long long)cblk * a.W;
+        const int wcols = (int)min((long long)a.W, a.d - cb);
+        OT* const out = static_cast<OT*>(a.out);
+        const int ahead = min(n, a.n_slots);
+        for (int j = 0; j < ahead; ++j) issue(b, j);
+        for (int j = 0; j < n; ++j) {
+            const int kind = __shfl_sync(0xFFFFFFFFu, b.kind, j);
+            const int y = __shfl_sync(0xFFFFFFFFu, b.y, j);
+            if (!mbar_wait(bars + 8u * (unsigned)cslot, (cphase >> cslot) & 1u, abort_flag)) { give_up(); return false; }
+            cphase ^= 1u << cslot;
+            issued_mask &= ~(1u << cslot);
+            const char* sp = ring_ptr + (size_t)cslot * a.slot_bytes;
+            if (kind & kUnitAdd) {
+                Acc<VC> v[K];
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const int c = col(k);
+                    zero(v[k]);
+                    if (c < wcols) load_elems(reinterpret_cast<const VT*>(sp) + c, v[k]);
+                }
+#pragma unroll
+                for (int k = 0; k < K; ++k) add(acc[k], v[k]);
+            }
+            if (kind & kUnitFinal) {
+                OT* orow = out + (long long)y * a.d + cb;
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const int c = col(k);
+                    if (c < wcols) {
+                        Acc<VC> dn;
+                        zero(dn);
+                        if (a.dense_in) load_elems(reinterpret_cast<const OT*>(sp) + c, dn);
+                        if (!(kind & kUnitCopy)) add(dn, acc[k]);
+                        store_out(orow + c, dn);
+                    }
+                    zero(acc[k]);
+                }
+            }
+            __syncwarp();                                 // every lane has read the slot
+            cslot = cslot + 1 == a.n_slots ? 0 : cslot + 1;
+            if (j + a.n_slots < n) issue(b, j + a.n_slots);   // refill it
+            if (kind & kUnitChunkEnd) {
+                finish_chunk(acc, y, cblk);
+#pragma unroll
+                for (int k = 0; k < K; ++k) zero(acc[k]);
+            }
+        }
+        return true;
+    }
+
+    __device__ bool do_chunk(int cid, int cblk) {
+        const ChunkDesc cd = a.chunkdesc[cid];
+        const long long cb = (long long)cblk * a.W;
+        const unsigned bytes = (unsigned)(min((long long)a.W, a.d - cb) * (long long)sizeof(VT));
+        Acc<VC> acc[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) zero(acc[k]);
+        for (int base = 0; base < cd.len; base += 32) {
+            const int q = base + lane;
+            UnitBlock b{nullptr, 0u, 0, cid};
+            if (q < cd.len) {
+                const unsigned p = a.perm[cd.begin + q];
+                if (p < (unsigned)a.n_total) { b.src = resolve_row<VT>(a, p) + cb; b.bytes = bytes; b.kind = kUnitAdd; }
+                if (q == cd.len - 1) b.kind |= kUnitChunkEnd;
+            }
+            if (!run_block(acc, b, min(32, cd.len - base), cblk)) return false;
+        }
+        return true;
+    }
+
+    // A batch of consecutive output rows: their entries and their closing units, flattened
+    __device__ bool do_rows(int batch, int cblk) {
+        const int2 bt = a.batches[batch];
+        if (bt.x == 0) return true;                       // no row starts in this batch
+        const int v0 = bt.x - 1;
+        const int nrows = min(bt.y - bt.x + 1, 31);
+        const long long cb = (long long)cblk * a.W;
+        const long long wcols = min((long long)a.W, a.d - cb);
+        int o = 0;
+        if (lane <= nrows) o = a.offsets[v0 + lane];
+        const int o_next = __shfl_down_sync(0xFFFFFFFFu, o, 1);
+        const int cnt = lane < nrows ? o_next - o : 0;
+        const int nunits = (lane < nrows && cnt <= a.chunk) ? cnt + 1 : 0;   // heavy rows belong to the chunk items
+        int incl = nunits;
+#pragma unroll
+        for (int s = 1; s < 32; s <<= 1) {
+            int t = __shfl_up_sync(0xFFFFFFFFu, incl, s);
+            if (lane >= s) incl += t;
+        }
+        const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        Acc<VC> acc[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) zero(acc[k]);
+        for (int base = 0; base < total; base += 32) {
+            const int q = base + lane;
+            int i = 0;                                   // row of unit q: rows whose units all come before q
+#pragma unroll
+            for (int step = 16; step > 0; step >>= 1)
+                if (__shfl_sync(0xFFFFFFFFu, incl, i + step - 1) <= q) i += step;
+            i = min(i, 31);
+            const int e = q - (__shfl_sync(0xFFFFFFFFu, incl, i) - __shfl_sync(0xFFFFFFFFu, nunits, i));
+            const int ci = __shfl_sync(0xFFFFFFFFu, cnt, i);
+            const int oi = __shfl_sync(0xFFFFFFFFu, o, i);
+            UnitBlock b{nullptr, 0u, 0, 0};
+            if (q < total) {
+                if (e < ci) {
+                    const unsigned p = a.perm[oi + e];
+                    if (p < (unsigned)a.n_total) {
+                        b.src = resolve_row<VT>(a, p) + cb;
+                        b.bytes = (unsigned)(wcols * (long long)sizeof(VT));
+                        b.kind = kUnitAdd;
+                    }
+                } else {
+                    b.y = v0 + i;
+                    b.kind = kUnitFinal | (ci == 0 ? kUnitCopy : 0);
+                    if (a.dense_in) {
+                        b.src = static_cast<const OT*>(a.dense_in) + (long long)b.y * a.d + cb;
+                        b.bytes = (unsigned)(wcols * (long long)sizeof(OT));
+                    }
+                }
+            }
+            if (!run_block(acc, b, min(32, total - base), cblk)) return false;
+        }
+        return true;
+    }
+
+    __device__ void run() {
+        const unsigned n_chunks = (unsigned)a.hdr->n_chunks;
+        const unsigned n_base = n_chunks + (unsigned)a.hdr->n_batches;
+        const unsigned n_items = n_base * (unsigned)a.ncb;
+        bool ok = true;
+        unsigned pending = 0;
+        if (lane == 0) pending = atomicAdd(&a.hdr->work_counter, 1u);
+        while (ok) {
+            const unsigned item = __shfl_sync(0xFFFFFFFFu, pending, 0);
+            if (item >= n_items) break;
+            if (lane == 0) pending = atomicAdd(&a.hdr->work_counter, 1u);   // in flight while this item is processed
+            const int cblk = (int)(item / n_base);
+            const unsigned base = item - (unsigned)cblk * n_base;
+            ok = base < n_chunks ? do_chunk((int)base, cblk) : do_rows((int)(base - n_chunks), cblk);
+        }
+        if (!ok) {
+            // a wait gave up: let every copy this warp has issued land before the CTA's shared memory goes away
+            for (int s = 0; s < a.n_slots; ++s) {
+                if (issued_mask & (1u << s)) {
+                    const long long start = clock64();
+                    while (!mbar_try_wait(bars + 8u * (unsigned)s, (cphase >> s) & 1u) && clock64() - start < kWaitCycles) {}
+                }
+            }
+        }
+    }
 };
 
 template <typename VT, typename OT, int K>
-__global__ void __launch_bounds__(kMainThreads)
-k_reduce_rows(const MainArgs a) {
-    RowReducer<VT, OT, K> rr(a);
-    const int n_chunks = a.hdr->n_chunks;
-    const unsigned n_items = (unsigned)n_chunks + (unsigned)((a.vocab + kRowsPerBatch - 1) / kRowsPerBatch);
-    if (blockIdx.x == 0 && threadIdx.x == 0 && a.result) a.result->status = a.hdr->status;
-    while (true) {
-        unsigned item = 0;
-        if (rr.lane == 0) item = atomicAdd(&a.hdr->work_counter, 1u);
-        item = __shfl_sync(0xFFFFFFFFu, item, 0);
-        if (item >= n_items) break;
-        if (item < (unsigned)n_chunks) rr.do_chunk((int)item);
-        else rr.do_row_batch((int)(item - (unsigned)n_chunks));
+__global__ void __launch_bounds__(kPipeThreads)
+k_reduce_rows(const __grid_constant__ MainArgs a) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ int s_abort;
+    unsigned long long* bar_base = reinterpret_cast<unsigned long long*>(smem_raw);
+    char* slot_base = reinterpret_cast<char*>(smem_raw) + kPipeHeaderReserve;
+    const int warp = warp_id();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPipeWarps * a.n_slots; ++s) mbar_init(smem_addr(&bar_base[s]), 1u);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    {
+        char* my_ring = slot_base + (size_t)warp * (size_t)a.n_slots * (size_t)a.slot_bytes;
+        WarpPipe<VT, OT, K> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort);
+        pipe.run();
+    }
+    __syncthreads();
+    // the last CTA to finish reports the status word (it may have been raised by this kernel)
+    if (threadIdx.x == 0 && a.result) {
+        __threadfence();
+        if (atomicAdd(&a.hdr->done, 1u) == gridDim.x - 1u) {
+            __threadfence();
+            a.result->status = *reinterpret_cast<volatile int*>(&a.hdr->status);
+        }
     }
 }
 
@@ -344,8 +500,16 @@ k_reduce_rows_scalar(const MainArgs a) {
     }
 }
 
+template <typename VT, typename OT, int K>
+static cudaError_t launch_pipe(const MainArgs& a, int grid, size_t smem, cudaStream_t stream) {
+    cudaError_t e = cudaFuncSetAttribute(k_reduce_rows<VT, OT, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_reduce_rows<VT, OT, K><<<grid, kPipeThreads, smem, stream>>>(a);
+    return cudaGetLastError();
+}
+
 template <typename VT, typename OT>
-static cudaError_t launch_typed(const MainArgs& a, bool vector_ok, int grid, cudaStream_t stream) {
+static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaStream_t stream) {
     if (!vector_ok) {
         long long total = (long long)a.vocab * a.d;
         long long blocks = (total + 255) / 256;
@@ -354,22 +518,23 @@ static cudaError_t launch_typed(const MainArgs& a, bool vector_ok, int grid, cud
         k_reduce_rows_scalar<VT, OT><<<(int)blocks, 256, 0, stream>>>(a);
         return cudaGetLastError();
     }
-    constexpr int VC = 16 / sizeof(VT);
-    const long long groups = (a.d + 32LL * VC - 1) / (32LL * VC);   // 16-byte groups per lane needed for one pass
+    const PipeShape ps = pipe_shape((int)sizeof(VT), (int)sizeof(OT), a.d);
+    a.W = ps.W; a.ncb = ps.ncb; a.slot_bytes = ps.slot_bytes; a.n_slots = ps.n_slots;
+    const size_t smem = size_t(kPipeHeaderReserve) + size_t(kPipeWarps) * size_t(ps.n_slots) * size_t(ps.slot_bytes);
+    const int grid = sm_count * ps.ctas_per_sm;
     constexpr int kMaxK = sizeof(VT) == 4 ? 8 : 4;
-    if (groups <= 1) k_reduce_rows<VT, OT, 1><<<grid, kMainThreads, 0, stream>>>(a);
-    else if (groups <= 2) k_reduce_rows<VT, OT, 2><<<grid, kMainThreads, 0, stream>>>(a);
-    else if (groups <= 4 || kMaxK == 4) k_reduce_rows<VT, OT, 4><<<grid, kMainThreads, 0, stream>>>(a);
-    else k_reduce_rows<VT, OT, kMaxK><<<grid, kMainThreads, 0, stream>>>(a);
-    return cudaGetLastError();
+    if (ps.K == 1) return launch_pipe<VT, OT, 1>(a, grid, smem, stream);
+    if (ps.K == 2) return launch_pipe<VT, OT, 2>(a, grid, smem, stream);
+    if (ps.K == 4 || kMaxK == 4) return launch_pipe<VT, OT, 4>(a, grid, smem, stream);
+    return launch_pipe<VT, OT, kMaxK>(a, grid, smem, stream);
 }
 
-cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int grid,
+cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,
                                cudaStream_t stream) {
-    if (value_type == DST_F32 && out_type == DST_F32) return launch_typed<float, float>(a, vector_ok, grid, stream);
-    if (value_type == DST_F32 && out_type == DST_BF16) return launch_typed<float, __nv_bfloat16>(a, vector_ok, grid, stream);
-    if (value_type == DST_BF16 && out_type == DST_F32) return launch_typed<__nv_bfloat16, float>(a, vector_ok, grid, stream);
-    return launch_typed<__nv_bfloat16, __nv_bfloat16>(a, vector_ok, grid, stream);
+    if (value_type == DST_F32 && out_type == DST_F32) return launch_typed<float, float>(a, vector_ok, sm_count, stream);
+    if (value_type == DST_F32 && out_type == DST_BF16) return launch_typed<float, __nv_bfloat16>(a, vector_ok, sm_count, stream);
+    if (value_type == DST_BF16 && out_type == DST_F32) return launch_typed<__nv_bfloat16, float>(a, vector_ok, sm_count, stream);
+    return launch_typed<__nv_bfloat16, __nv_bfloat16>(a, vector_ok, sm_count, stream);
 }
 
 }  // namespace dst
