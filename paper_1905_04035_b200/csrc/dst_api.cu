@@ -78,7 +78,7 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
 
     if (cudaMemsetAsync(ws, 0, L.zero_bytes, stream) != cudaSuccess) return DST_ERR_CUDA;
 
-    // a1/a2: histogram, at most kHistSlices slices per launch
+    // a1: validate and narrow, at most kHistSlices slices per launch
     int64_t start = 0;
     for (int first = 0; first < R; first += kHistSlices) {
         HistParams P;
@@ -92,28 +92,31 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
             start += s.n_rows;
             if (s.n_rows > longest) longest = s.n_rows;
         }
-        int grid_x = int((longest + kTile - 1) / kTile);
+        int grid_x = int((longest + kPrepTile - 1) / kPrepTile);
         if (grid_x < 1) grid_x = 1;   // still writes the slice table
-        if (launch_hist(P, grid_x, opts->index_type, hdr, count, digit, keys[0], tab, vocab, L.passes, stream) != cudaSuccess)
+        if (launch_prep(P, grid_x, opts->index_type, hdr, digit, keys[0], tab, vocab, L.passes, stream) != cudaSuccess)
+            return DST_ERR_CUDA;
+        ++g_launches;
+    }
+    if (n_total > 0) {
+        // a4: least significant digit first; keys/positions ping-pong between two buffers
+        for (int p = 0; p < L.passes; ++p) {
+            if (launch_radix_pass(int(L.n_tiles), hdr, keys[p & 1], p == 0 ? nullptr : pos[p & 1], keys[(p + 1) & 1],
+                                  pos[(p + 1) & 1], digit + p * 256, desc + size_t(p) * size_t(L.n_tiles) * 256, p,
+                                  int(n_total), stream) != cudaSuccess)
+                return DST_ERR_CUDA;
+            ++g_launches;
+        }
+        // a2: run lengths of the sorted keys
+        if (launch_bounds(hdr, keys[L.passes & 1], count, int(n_total), int(vocab), stream) != cudaSuccess)
             return DST_ERR_CUDA;
         ++g_launches;
     }
     // a3/a5/a6
-    if (launch_scan(opts->index_type, hdr, count, offsets, heavy, chunkdesc, unique_rows, counts, result,
-                    batches, int(vocab), int(L.vocab_pad), L.chunk, L.batch_units, stream) != cudaSuccess)
-        return DST_ERR_CUDA;
+    ScanParams sp{hdr, count, offsets, heavy, chunkdesc, unique_rows, counts, result, batches,
+                  reinterpret_cast<int*>(ws + L.off_scandesc), int(vocab), int(L.vocab_pad), L.chunk, L.batch_units};
+    if (launch_scan(opts->index_type, sp, stream) != cudaSuccess) return DST_ERR_CUDA;
     ++g_launches;
-    // a4: least significant digit first; keys/positions ping-pong between two buffers
-    if (n_total > 0) {
-        for (int p = 0; p < L.passes; ++p) {
-            const bool last = p == L.passes - 1;
-            if (launch_radix_pass(int(L.n_tiles), hdr, keys[p & 1], p == 0 ? nullptr : pos[p & 1],
-                                  last ? nullptr : keys[(p + 1) & 1], pos[(p + 1) & 1], digit + p * 256,
-                                  desc + size_t(p) * size_t(L.n_tiles) * 256, p, int(n_total), stream) != cudaSuccess)
-                return DST_ERR_CUDA;
-            ++g_launches;
-        }
-    }
     // a7/a8
     MainArgs a;
     a.hdr = hdr; a.offsets = offsets; a.perm = pos[L.passes & 1]; a.tab = tab; a.heavy = heavy;

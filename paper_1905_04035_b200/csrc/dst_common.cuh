@@ -11,9 +11,10 @@ namespace dst {
 
 // ---- fixed shape parameters -------------------------------------------------
 constexpr int kSortThreads = 256;           // threads of the histogram and radix-pass kernels
-constexpr int kSortItems = 8;               // keys per thread
-constexpr int kTile = kSortThreads * kSortItems;  // 2048 keys per CTA
-constexpr int kHashSlots = 4096;            // per-CTA key aggregation table (> kTile distinct keys never happen)
+constexpr int kSortItems = 16;              // keys per thread of a radix pass
+constexpr int kTile = kSortThreads * kSortItems;  // 4096 keys per CTA
+constexpr int kPrepItems = 8;               // indices per thread of the validation kernel
+constexpr int kPrepTile = kSortThreads * kPrepItems;
 constexpr int kMaxPasses = 4;               // 8-bit digits, keys below 2^31
 constexpr int kFanIn = 16;                  // children per node of the heavy-row combine tree
 constexpr int kMaxBatchUnits = 31;          // a light work item holds rows worth at most this many units (+ one row)
@@ -26,8 +27,9 @@ constexpr int kPipeHeaderReserve = 1024;    // mbarriers in front of the slots
 constexpr int kMaxBlockCols = 1024;         // columns per column block (32 fp32 accumulators per lane)
 constexpr int kSmemPerSm = 227 * 1024;
 constexpr long long kWaitCycles = 1LL << 31; // SM clock cycles (about a second) before an mbarrier wait gives up
-constexpr int kScanThreads = 1024;
-constexpr int kScanItems = 16;              // counters per thread and round in the scan kernel
+constexpr int kScanThreads = 256;
+constexpr int kScanItems = 8;               // rows per thread in the scan kernel
+constexpr int kScanTile = kScanThreads * kScanItems;
 constexpr int kSmCount = 148;               // B200; only used to pick the chunk length
 constexpr unsigned kInvalidKey = 0xFFFFFFFFu;
 constexpr unsigned kFlagMask = 0xC0000000u, kFlagAggregate = 0x40000000u, kFlagPrefix = 0x80000000u;
@@ -50,7 +52,8 @@ struct WsHeader {          // zeroed at the start of every call
     unsigned int ticket[kMaxPasses];
     unsigned int work_counter;
     int n_batches;         // light work items (row batches)
-    unsigned int pad1[2];
+    unsigned int scan_ticket;
+    unsigned int scan_done;
 };
 static_assert(sizeof(WsHeader) == 72, "header layout");
 
@@ -86,7 +89,7 @@ struct Layout {
     int64_t n_rows, vocab, d;
     int R, chunk, passes, batch_units;
     int64_t n_tiles, vocab_pad, heavy_max, chunk_max, upper_max, batch_max;
-    size_t off_header, off_count, off_digit, off_desc, off_nodecnt, off_batches, zero_bytes;
+    size_t off_header, off_count, off_digit, off_desc, off_nodecnt, off_batches, off_scandesc, zero_bytes;
     size_t off_offsets, off_keys[2], off_pos[2], off_tab, off_heavy, off_chunkdesc, off_partials;
     size_t total;
 };
@@ -168,6 +171,7 @@ inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab, i
     L.off_desc = take(size_t(L.passes) * size_t(L.n_tiles) * 256 * 4);
     L.off_nodecnt = take(size_t(L.upper_max) * size_t(pipe_shape(value_size, out_size, d).ncb) * 4);
     L.off_batches = take(size_t(L.batch_max) * 8);
+    L.off_scandesc = take(size_t((L.vocab_pad + kScanTile - 1) / kScanTile + 1) * 64);
     L.zero_bytes = o;
     L.off_offsets = take(size_t(L.vocab_pad + kScanItems) * 4);
     L.off_keys[0] = take(size_t(n_rows) * 4);
@@ -183,15 +187,27 @@ inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab, i
 }
 
 // ---- kernel launchers (defined next to their kernels) ----------------------------
-cudaError_t launch_hist(const HistParams& P, int grid_x, int index_type, WsHeader* hdr, unsigned* count,
-                        unsigned* digit_hist, unsigned* keys, SliceEntry* tab, long long vocab, int passes,
-                        cudaStream_t stream);
-cudaError_t launch_scan(int index_type, WsHeader* hdr, const unsigned* count, int* offsets, HeavyInfo* heavy,
-                        ChunkDesc* chunkdesc, void* unique_rows, int* counts_out, dst_result_t* result,
-                        int2* batches, int vocab, int vocab_pad, int chunk, int batch_units, cudaStream_t stream);
+struct ScanParams {
+    WsHeader* hdr;
+    const unsigned* count;
+    int* offsets;
+    HeavyInfo* heavy;
+    ChunkDesc* chunkdesc;
+    void* unique_rows;
+    int* counts_out;
+    dst_result_t* result;
+    int2* batches;
+    int* scan_desc;
+    int vocab, vocab_pad, chunk, batch_units;
+};
+cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeader* hdr, unsigned* digit_hist,
+                        unsigned* keys, SliceEntry* tab, long long vocab, int passes, cudaStream_t stream);
 cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
                               unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
                               int pass, int capacity, cudaStream_t stream);
+cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
+                          cudaStream_t stream);
+cudaError_t launch_scan(int index_type, const ScanParams& p, cudaStream_t stream);
 cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,
                                cudaStream_t stream);
 

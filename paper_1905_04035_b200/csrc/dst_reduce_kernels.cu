@@ -464,7 +464,8 @@ k_reduce_rows(const __grid_constant__ MainArgs a) {
     {
         char* my_ring = slot_base + (size_t)warp * (size_t)a.n_slots * (size_t)a.slot_bytes;
         WarpPipe<VT, OT, K> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort);
-        pipe.run();
+        // after a failed wait in an earlier kernel the tables are not to be trusted: touch nothing
+        if (*reinterpret_cast<volatile int*>(&a.hdr->status) != DST_ERR_TIMEOUT) pipe.run();
     }
     __syncthreads();
     // the last CTA to finish reports the status word (it may have been raised by this kernel)
