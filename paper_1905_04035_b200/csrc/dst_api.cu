@@ -66,7 +66,6 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     unsigned* pos[2] = {reinterpret_cast<unsigned*>(ws + L.off_pos[0]), reinterpret_cast<unsigned*>(ws + L.off_pos[1])};
     SliceEntry* tab = reinterpret_cast<SliceEntry*>(ws + L.off_tab);
     HeavyInfo* heavy = reinterpret_cast<HeavyInfo*>(ws + L.off_heavy);
-    ChunkDesc* chunkdesc = reinterpret_cast<ChunkDesc*>(ws + L.off_chunkdesc);
     float* partials = reinterpret_cast<float*>(ws + L.off_partials);
 
     // the fast kernels need 16-byte aligned rows everywhere
@@ -78,49 +77,67 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
 
     if (cudaMemsetAsync(ws, 0, L.zero_bytes, stream) != cudaSuccess) return DST_ERR_CUDA;
 
-    // a1: validate and narrow, at most kHistSlices slices per launch
-    int64_t start = 0;
-    for (int first = 0; first < R; first += kHistSlices) {
+    const unsigned* perm = pos[L.passes & 1];
+    if (n_total > 0 && n_total <= kSmallMaxRows && vocab <= 65536 && R <= kHistSlices) {
+        // small input: validation, both radix passes and the run lengths in one CTA
         HistParams P;
         memset(&P, 0, sizeof P);
-        P.n = R - first < kHistSlices ? R - first : kHistSlices;
-        P.first = first;
-        int64_t longest = 0;
-        for (int i = 0; i < P.n; ++i) {
-            const dst_slice_t& s = slices[first + i];
-            P.s[i] = SliceEntry{s.indices, s.values, (long long)start, (long long)s.n_rows};
-            start += s.n_rows;
-            if (s.n_rows > longest) longest = s.n_rows;
+        P.n = R;
+        int64_t start = 0;
+        for (int i = 0; i < R; ++i) {
+            P.s[i] = SliceEntry{slices[i].indices, slices[i].values, (long long)start, (long long)slices[i].n_rows};
+            start += slices[i].n_rows;
         }
-        int grid_x = int((longest + kPrepTile - 1) / kPrepTile);
-        if (grid_x < 1) grid_x = 1;   // still writes the slice table
-        if (launch_prep(P, grid_x, opts->index_type, hdr, digit, keys[0], tab, vocab, L.passes, stream) != cudaSuccess)
+        if (launch_sort_small(P, opts->index_type, hdr, tab, keys[0], pos[0], count, int(n_total), vocab, stream) !=
+            cudaSuccess)
             return DST_ERR_CUDA;
         ++g_launches;
-    }
-    if (n_total > 0) {
-        // a4: least significant digit first; keys/positions ping-pong between two buffers
-        for (int p = 0; p < L.passes; ++p) {
-            if (launch_radix_pass(int(L.n_tiles), hdr, keys[p & 1], p == 0 ? nullptr : pos[p & 1], keys[(p + 1) & 1],
-                                  pos[(p + 1) & 1], digit + p * 256, desc + size_t(p) * size_t(L.n_tiles) * 256, p,
-                                  int(n_total), stream) != cudaSuccess)
+        perm = pos[0];
+    } else {
+        // a1: validate and narrow, at most kHistSlices slices per launch
+        int64_t start = 0;
+        for (int first = 0; first < R; first += kHistSlices) {
+            HistParams P;
+            memset(&P, 0, sizeof P);
+            P.n = R - first < kHistSlices ? R - first : kHistSlices;
+            P.first = first;
+            int64_t longest = 0;
+            for (int i = 0; i < P.n; ++i) {
+                const dst_slice_t& s = slices[first + i];
+                P.s[i] = SliceEntry{s.indices, s.values, (long long)start, (long long)s.n_rows};
+                start += s.n_rows;
+                if (s.n_rows > longest) longest = s.n_rows;
+            }
+            int grid_x = int((longest + kPrepTile - 1) / kPrepTile);
+            if (grid_x < 1) grid_x = 1;   // still writes the slice table
+            if (launch_prep(P, grid_x, opts->index_type, hdr, digit, keys[0], tab, vocab, L.passes, stream) != cudaSuccess)
                 return DST_ERR_CUDA;
             ++g_launches;
         }
-        // a2: run lengths of the sorted keys
-        if (launch_bounds(hdr, keys[L.passes & 1], count, int(n_total), int(vocab), stream) != cudaSuccess)
-            return DST_ERR_CUDA;
-        ++g_launches;
+        if (n_total > 0) {
+            // a4: least significant digit first; keys/positions ping-pong between two buffers
+            for (int p = 0; p < L.passes; ++p) {
+                if (launch_radix_pass(int(L.n_tiles), hdr, keys[p & 1], p == 0 ? nullptr : pos[p & 1], keys[(p + 1) & 1],
+                                      pos[(p + 1) & 1], digit + p * 256, desc + size_t(p) * size_t(L.n_tiles) * 256, p,
+                                      int(n_total), stream) != cudaSuccess)
+                    return DST_ERR_CUDA;
+                ++g_launches;
+            }
+            // a2: run lengths of the sorted keys
+            if (launch_bounds(hdr, keys[L.passes & 1], count, int(n_total), int(vocab), stream) != cudaSuccess)
+                return DST_ERR_CUDA;
+            ++g_launches;
+        }
     }
     // a3/a5/a6
-    ScanParams sp{hdr, count, offsets, heavy, chunkdesc, unique_rows, counts, result, batches,
+    ScanParams sp{hdr, count, offsets, heavy, unique_rows, counts, result, batches,
                   reinterpret_cast<int*>(ws + L.off_scandesc), int(vocab), int(L.vocab_pad), L.chunk, L.batch_units};
     if (launch_scan(opts->index_type, sp, stream) != cudaSuccess) return DST_ERR_CUDA;
     ++g_launches;
     // a7/a8
     MainArgs a;
-    a.hdr = hdr; a.offsets = offsets; a.perm = pos[L.passes & 1]; a.tab = tab; a.heavy = heavy;
-    a.chunkdesc = chunkdesc; a.batches = batches; a.node_cnt = nodecnt; a.partials = partials; a.dense_in = dense_in; a.out = out;
+    a.hdr = hdr; a.offsets = offsets; a.perm = perm; a.tab = tab; a.heavy = heavy;
+    a.batches = batches; a.node_cnt = nodecnt; a.partials = partials; a.dense_in = dense_in; a.out = out;
     a.result = result; a.d = d; a.vocab = int(vocab); a.n_total = int(n_total); a.R = R; a.chunk = L.chunk;
     a.chunk_max = int(L.chunk_max); a.upper_max = int(L.upper_max);
     a.W = a.ncb = a.slot_bytes = a.n_slots = 0;   // set by the launcher

@@ -13,6 +13,9 @@ namespace dst {
 constexpr int kSortThreads = 256;           // threads of the histogram and radix-pass kernels
 constexpr int kSortItems = 16;              // keys per thread of a radix pass
 constexpr int kTile = kSortThreads * kSortItems;  // 4096 keys per CTA
+constexpr int kSmallThreads = 1024;          // the one-CTA sort for small inputs
+constexpr int kSmallGroups = 32;            // groups of 32 entries per warp (at most)
+constexpr int kSmallMaxRows = kSmallThreads * kSmallGroups;   // 32768
 constexpr int kPrepItems = 8;               // indices per thread of the validation kernel
 constexpr int kPrepTile = kSortThreads * kPrepItems;
 constexpr int kMaxPasses = 4;               // 8-bit digits, keys below 2^31
@@ -76,9 +79,13 @@ struct HeavyInfo {         // a row whose segment is split into chunks
     int chunk_base;        // id of its first chunk
     int upper_base;        // id of its first upper tree node
     int n_chunks;
+    int begin;             // first entry of its segment in perm[]
+    int count;             // entries in its segment
+    int pad[2];
 };
+static_assert(sizeof(HeavyInfo) == 32, "heavy-row record layout");
 
-struct ChunkDesc {         // one chunk work item
+struct ChunkDesc {         // one chunk work item (derived from HeavyInfo on the fly)
     int row;
     int begin;             // first entry in perm[]
     int len;
@@ -90,7 +97,7 @@ struct Layout {
     int R, chunk, passes, batch_units;
     int64_t n_tiles, vocab_pad, heavy_max, chunk_max, upper_max, batch_max;
     size_t off_header, off_count, off_digit, off_desc, off_nodecnt, off_batches, off_scandesc, zero_bytes;
-    size_t off_offsets, off_keys[2], off_pos[2], off_tab, off_heavy, off_chunkdesc, off_partials;
+    size_t off_offsets, off_keys[2], off_pos[2], off_tab, off_heavy, off_partials;
     size_t total;
 };
 
@@ -101,7 +108,6 @@ struct MainArgs {
     const unsigned* perm;
     const SliceEntry* tab;
     const HeavyInfo* heavy;
-    const ChunkDesc* chunkdesc;
     const int2* batches;   // per row batch: first row + 1 (0: empty batch), last row + 1
     unsigned* node_cnt;
     float* partials;
@@ -180,7 +186,6 @@ inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab, i
     L.off_pos[1] = take(size_t(n_rows) * 4);
     L.off_tab = take(size_t(R > 0 ? R : 1) * sizeof(SliceEntry));
     L.off_heavy = take(size_t(L.heavy_max + 1) * sizeof(HeavyInfo));
-    L.off_chunkdesc = take(size_t(L.chunk_max + 1) * sizeof(ChunkDesc));
     L.off_partials = take(size_t(L.chunk_max + L.upper_max) * size_t(d) * 4);
     L.total = o;
     return L;
@@ -192,7 +197,6 @@ struct ScanParams {
     const unsigned* count;
     int* offsets;
     HeavyInfo* heavy;
-    ChunkDesc* chunkdesc;
     void* unique_rows;
     int* counts_out;
     dst_result_t* result;
@@ -205,6 +209,8 @@ cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeade
 cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
                               unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
                               int pass, int capacity, cudaStream_t stream);
+cudaError_t launch_sort_small(const HistParams& P, int index_type, WsHeader* hdr, SliceEntry* tab, unsigned* skeys,
+                              unsigned* perm, unsigned* count, int n_total, long long vocab, cudaStream_t stream);
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
                           cudaStream_t stream);
 cudaError_t launch_scan(int index_type, const ScanParams& p, cudaStream_t stream);

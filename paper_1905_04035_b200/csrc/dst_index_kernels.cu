@@ -210,7 +210,6 @@ struct ScanArgs {
     const unsigned* count;
     int* offsets;
     HeavyInfo* heavy;
-    ChunkDesc* chunkdesc;
     void* unique_rows;
     int* counts_out;
     dst_result_t* result;
@@ -219,8 +218,6 @@ struct ScanArgs {
     int vocab, vocab_pad, chunk, batch_units, n_tiles;
 };
 
-constexpr int kBigRows = 256;       // heavy rows per tile whose chunk descriptors the whole CTA writes together
-constexpr int kInlineChunks = 4;    // heavy rows with at most this many chunks are described by one thread
 
 __device__ __forceinline__ int row_units(int cc, int chunk) { return cc > chunk ? 1 : cc + 1; }
 
@@ -263,9 +260,6 @@ k_scan(const ScanArgs s) {
     __shared__ int s_nearest;
     __shared__ int s_tile;
     __shared__ int s_fail;
-    __shared__ int4 s_big[kBigRows];     // row, first entry, count, first chunk id
-    __shared__ int s_bigh[kBigRows];     // index into heavy[]
-    __shared__ int s_nbig;
     WsHeader* hdr = s.hdr;
     const int chunk = s.chunk, B = s.batch_units, vocab = s.vocab;
     IT* unique_rows = static_cast<IT*>(s.unique_rows);
@@ -273,7 +267,7 @@ k_scan(const ScanArgs s) {
         s_tile = (int)atomicAdd(&hdr->scan_ticket, 1u);   // tiles start in id order
         // after a failed look-back count[] is not to be trusted: leave every table empty
         if (*reinterpret_cast<volatile int*>(&hdr->status) == DST_ERR_TIMEOUT) s_tile = -1;
-        s_nbig = 0; s_fail = 0; s_nearest = 0x7FFFFFFF;
+        s_fail = 0; s_nearest = 0x7FFFFFFF;
     }
     if (threadIdx.x < 6) s_prefix[threadIdx.x] = 0;
     __syncthreads();
@@ -378,16 +372,7 @@ k_scan(const ScanArgs s) {
             if (cc > chunk) {
                 // a6: a heavy row becomes n chunk items and a combine tree
                 const int n = (cc + chunk - 1) / chunk;
-                const int h = run.v[2];
-                s.heavy[h] = HeavyInfo{v, run.v[3], run.v[4], n};
-                const int slot = n > kInlineChunks ? atomicAdd(&s_nbig, 1) : kBigRows;
-                if (slot < kBigRows) {
-                    s_big[slot] = make_int4(v, run.v[0], cc, run.v[3]);
-                    s_bigh[slot] = h;
-                } else {
-                    for (int k = 0; k < n; ++k)
-                        s.chunkdesc[run.v[3] + k] = ChunkDesc{v, run.v[0] + k * chunk, min(chunk, cc - k * chunk), h};
-                }
+                s.heavy[run.v[2]] = HeavyInfo{v, run.v[3], run.v[4], n, run.v[0], cc, {0, 0}};
                 run.v[2] += 1; run.v[3] += n; run.v[4] += upper_nodes(n);
             }
             run.v[0] += cc;
@@ -404,16 +389,6 @@ k_scan(const ScanArgs s) {
         int4* dst = reinterpret_cast<int4*>(s.offsets + e0);
 #pragma unroll
         for (int q = 0; q < kScanItems / 4; ++q) dst[q] = make_int4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
-    }
-    // chunk descriptors of the rows with many chunks, all threads together
-    __syncthreads();
-    const int nbig = min(s_nbig, kBigRows);
-    for (int r = 0; r < nbig; ++r) {
-        const int4 bg = s_big[r];
-        const int h = s_bigh[r];
-        const int n = (bg.z + chunk - 1) / chunk;
-        for (int k = threadIdx.x; k < n; k += kScanThreads)
-            s.chunkdesc[bg.w + k] = ChunkDesc{bg.x, bg.y + k * chunk, min(chunk, bg.z - k * chunk), h};
     }
     for (int o = 16; o > 0; o >>= 1) maxseg = max(maxseg, __shfl_down_sync(0xFFFFFFFFu, maxseg, o));
     if (lane_id() == 0 && maxseg > 0) atomicMax(&hdr->max_segment, maxseg);
@@ -444,6 +419,133 @@ k_scan(const ScanArgs s) {
     }
 }
 
+// ---------------------------------------------------------------------------
+// Small inputs: a1 + a4 + a2 in one CTA.  The keys stay on chip between the two radix passes
+// (registers, then one packed word per entry in shared memory), so there is no look-back and no
+// intermediate global traffic.  Needs n_total <= kSmallMaxRows, vocab <= 65536, R <= kHistSlices.
+//
+// Warp w owns the entries [w * L, (w + 1) * L) in input order and walks them 32 at a time, so
+// ranking inside a warp by lane order and across warps by warp order is stable.
+// ---------------------------------------------------------------------------
+struct SmallRank {
+    // one group of 32 entries: add the group to the warp's running digit counters and return
+    // this lane's rank among the entries of the tile with the same digit (wh: this warp's row)
+    static __device__ __forceinline__ unsigned step(unsigned short* wh, bool valid, unsigned dg, int lane) {
+        const unsigned m = __match_any_sync(0xFFFFFFFFu, valid ? dg : (0x10000u | lane));
+        const int leader = __ffs(m) - 1;
+        unsigned pre = 0;
+        if (valid && lane == leader) { pre = wh[dg]; wh[dg] = (unsigned short)(pre + __popc(m)); }
+        pre = __shfl_sync(0xFFFFFFFFu, pre, leader);
+        __syncwarp();
+        return pre + __popc(m & ((1u << lane) - 1u));
+    }
+};
+
+// wh[w][d] holds per-warp digit counts: turn them into the position of the first entry of
+// (digit d, warp w) in the sorted order; returns the number of entries (valid at thread 255)
+__device__ __forceinline__ unsigned small_bases(unsigned short (*wh)[256], unsigned* s_warp_tot) {
+    const int lane = lane_id(), warp = warp_id();
+    unsigned tot = 0;
+    if (threadIdx.x < 256) {
+#pragma unroll 8
+        for (int w = 0; w < kSmallThreads / 32; ++w) { unsigned t = wh[w][threadIdx.x]; wh[w][threadIdx.x] = (unsigned short)tot; tot += t; }
+    }
+    unsigned inc = tot;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { unsigned t = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t; }
+    if (lane == 31 && warp < 8) s_warp_tot[warp] = inc;
+    __syncthreads();
+    unsigned n_all = 0;
+    if (threadIdx.x < 256) {
+        unsigned base = inc - tot;
+        for (int w = 0; w < warp; ++w) base += s_warp_tot[w];
+#pragma unroll 8
+        for (int w = 0; w < kSmallThreads / 32; ++w) wh[w][threadIdx.x] = (unsigned short)(wh[w][threadIdx.x] + base);
+        n_all = base + tot;
+    }
+    __syncthreads();
+    return n_all;
+}
+
+template <typename IT>
+__global__ void __launch_bounds__(kSmallThreads)
+k_sort_small(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, SliceEntry* __restrict__ tab,
+             unsigned* __restrict__ skeys, unsigned* __restrict__ perm, unsigned* __restrict__ count, int n_total,
+             long long vocab) {
+    extern __shared__ unsigned packed[];             // pass 0 output: key << 16 | position
+    __shared__ unsigned short wh[kSmallThreads / 32][256];
+    __shared__ unsigned s_warp_tot[8];
+    __shared__ int s_nvalid;
+    const int lane = lane_id(), warp = warp_id();
+    if (threadIdx.x < P.n) tab[P.first + threadIdx.x] = P.s[threadIdx.x];
+    for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(wh[warp])[s] = 0;
+
+    // ---- load and validate: warp `warp` owns entries [warp * L, warp * L + L)
+    const int L = ((n_total + kSmallThreads - 1) / kSmallThreads) * 32;
+    const int ng = L / 32;                           // groups per warp, <= kSmallGroups
+    unsigned key[kSmallGroups];
+    {
+        int r = 0;
+#pragma unroll
+        for (int g = 0; g < kSmallGroups; ++g) {
+            key[g] = kInvalidKey;
+            const int e = warp * L + g * 32 + lane;
+            if (g < ng && e < n_total) {
+                while (r + 1 < P.n && (long long)e >= P.s[r + 1].start) ++r;
+                const long long v = (long long)static_cast<const IT*>(P.s[r].indices)[(long long)e - P.s[r].start];
+                if (v >= 0 && v < vocab) key[g] = (unsigned)v;
+            }
+        }
+    }
+    __syncwarp();
+    // ---- pass 0: low digit, registers -> shared
+#pragma unroll
+    for (int g = 0; g < kSmallGroups; ++g)
+        if (g < ng) SmallRank::step(wh[warp], key[g] != kInvalidKey, key[g] & 255u, lane);
+    __syncthreads();
+    const unsigned n_all = small_bases(wh, s_warp_tot);
+    if (threadIdx.x == 255) s_nvalid = (int)n_all;
+#pragma unroll
+    for (int g = 0; g < kSmallGroups; ++g) {
+        if (g < ng) {
+            const bool valid = key[g] != kInvalidKey;
+            const unsigned q = SmallRank::step(wh[warp], valid, key[g] & 255u, lane);
+            if (valid) packed[q] = (key[g] << 16) | (unsigned)(warp * L + g * 32 + lane);
+        }
+    }
+    __syncthreads();
+    const int n_valid = s_nvalid;
+    // ---- pass 1: high digit, shared -> global
+    for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(wh[warp])[s] = 0;
+    __syncwarp();
+    const int L1 = ((n_valid + kSmallThreads - 1) / kSmallThreads) * 32;
+    for (int g = 0; g < L1 / 32; ++g) {
+        const int e = warp * L1 + g * 32 + lane;
+        const bool valid = e < n_valid;
+        const unsigned x = valid ? packed[e] : 0u;
+        SmallRank::step(wh[warp], valid, x >> 24, lane);
+    }
+    __syncthreads();
+    small_bases(wh, s_warp_tot);
+    for (int g = 0; g < L1 / 32; ++g) {
+        const int e = warp * L1 + g * 32 + lane;
+        const bool valid = e < n_valid;
+        const unsigned x = valid ? packed[e] : 0u;
+        const unsigned q = SmallRank::step(wh[warp], valid, x >> 24, lane);
+        if (valid) { perm[q] = x & 0xFFFFu; skeys[q] = x >> 16; }
+    }
+    __syncthreads();
+    // ---- a2: run lengths of the sorted keys (see k_bounds)
+    for (int i = threadIdx.x; i < n_valid; i += kSmallThreads) {
+        const unsigned k = skeys[i];
+        const unsigned prev = i > 0 ? skeys[i - 1] : ~k;
+        const unsigned next = i + 1 < n_valid ? skeys[i + 1] : ~k;
+        if (prev != k) atomicSub(&count[k], (unsigned)i);
+        if (next != k) atomicAdd(&count[k], (unsigned)i + 1u);
+    }
+    if (threadIdx.x == 0) hdr->n_bad = (unsigned long long)(n_total - n_valid);
+}
+
 // ---- host-side launchers ------------------------------------------------------
 cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeader* hdr, unsigned* digit_hist,
                         unsigned* keys, SliceEntry* tab, long long vocab, int passes, cudaStream_t stream) {
@@ -463,6 +565,22 @@ cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_key
     return cudaGetLastError();
 }
 
+cudaError_t launch_sort_small(const HistParams& P, int index_type, WsHeader* hdr, SliceEntry* tab, unsigned* skeys,
+                              unsigned* perm, unsigned* count, int n_total, long long vocab, cudaStream_t stream) {
+    const size_t smem = size_t(n_total) * 4;
+    cudaError_t e;
+    if (index_type == DST_I64) {
+        e = cudaFuncSetAttribute(k_sort_small<long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmallMaxRows * 4);
+        if (e != cudaSuccess) return e;
+        k_sort_small<long long><<<1, kSmallThreads, smem, stream>>>(P, hdr, tab, skeys, perm, count, n_total, vocab);
+    } else {
+        e = cudaFuncSetAttribute(k_sort_small<int>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmallMaxRows * 4);
+        if (e != cudaSuccess) return e;
+        k_sort_small<int><<<1, kSmallThreads, smem, stream>>>(P, hdr, tab, skeys, perm, count, n_total, vocab);
+    }
+    return cudaGetLastError();
+}
+
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
                           cudaStream_t stream) {
     k_bounds<<<(capacity + 255) / 256, 256, 0, stream>>>(hdr, keys, count, capacity, vocab);
@@ -471,7 +589,7 @@ cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* c
 
 cudaError_t launch_scan(int index_type, const ScanParams& p, cudaStream_t stream) {
     const int n_tiles = (p.vocab_pad + kScanTile - 1) / kScanTile;
-    ScanArgs s{p.hdr, p.count, p.offsets, p.heavy, p.chunkdesc, p.unique_rows, p.counts_out, p.result, p.batches,
+    ScanArgs s{p.hdr, p.count, p.offsets, p.heavy, p.unique_rows, p.counts_out, p.result, p.batches,
                p.scan_desc, p.vocab, p.vocab_pad, p.chunk, p.batch_units, n_tiles};
     if (index_type == DST_I64) k_scan<long long><<<n_tiles, kScanThreads, 0, stream>>>(s);
     else k_scan<int><<<n_tiles, kScanThreads, 0, stream>>>(s);

@@ -226,9 +226,31 @@ struct WarpPipe {
         }
     }
 
+    // Heavy row that owns chunk cid: the last h with heavy[h].chunk_base <= cid.  All lanes probe
+    // at once, so the table (a few hundred entries) is searched in two or three steps.
+    __device__ __forceinline__ int find_heavy(int cid) const {
+        int lo = 0, hi = a.hdr->n_heavy;
+        while (hi - lo > 1) {
+            const int step = (hi - lo + 31) / 32;
+            const int idx = lo + lane * step;
+            const bool le = idx < hi && __ldg(&a.heavy[idx].chunk_base) <= cid;
+            const int t = __popc(__ballot_sync(0xFFFFFFFFu, le));      // lane 0 always qualifies
+            lo += (t - 1) * step;
+            hi = min(hi, lo + step);
+        }
+        return lo;
+    }
+    __device__ __forceinline__ ChunkDesc chunk_of(int cid) const {
+        const int h = find_heavy(cid);
+        const HeavyInfo hi = a.heavy[h];
+        const int k = cid - hi.chunk_base;
+        return ChunkDesc{hi.row, hi.begin + k * a.chunk, min(a.chunk, hi.count - k * a.chunk), h};
+    }
+
     // The chunk's sum is in acc: store it as a partial row and climb the combine tree while this
     // warp is the last child to arrive.
     __device__ void finish_chunk(Acc<VC> (&acc)[K], int cid, int cblk) const {
+        const HeavyInfo hi = a.heavy[find_heavy(cid)];
         const long long cb = (long long)cblk * a.W;
         const int wcols = (int)min((long long)a.W, a.d - cb);
         {
@@ -239,8 +261,6 @@ struct WarpPipe {
                 if (c < wcols) store_partial(pr + c, acc[k]);
             }
         }
-        const ChunkDesc cd = a.chunkdesc[cid];
-        const HeavyInfo hi = a.heavy[cd.heavy];
         unsigned* node_cnt = a.node_cnt + (size_t)cblk * (size_t)a.upper_max;
         int j = cid - hi.chunk_base;     // index inside the current level
         int n_level = hi.n_chunks;       // nodes on the current level
@@ -345,7 +365,7 @@ struct WarpPipe {
     }
 
     __device__ bool do_chunk(int cid, int cblk) {
-        const ChunkDesc cd = a.chunkdesc[cid];
+        const ChunkDesc cd = chunk_of(cid);
         const long long cb = (long long)cblk * a.W;
         const unsigned bytes = (unsigned)(min((long long)a.W, a.d - cb) * (long long)sizeof(VT));
         Acc<VC> acc[K];
