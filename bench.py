@@ -207,6 +207,54 @@ def time_device(prob: DeviceProblem, steps: int, warmup: int, dist_ctx=None, clo
     return total_ms, kernel_ms, launches, clock_info
 
 
+def time_device_graph(prob: DeviceProblem, steps: int, warmup: int, dist_ctx=None, clocks: ClockSampler = None):
+    """The same K steps, each step replayed from a CUDA graph captured once per buffer set (the library
+    allocates nothing and never synchronises, so a call can be captured as it is).  Returns total ms."""
+    import torch
+    import paper_1905_04035_b200 as dst
+    prob.step(0)                       # first call outside capture (sets kernel attributes)
+    torch.cuda.synchronize()
+    graphs = []
+    for slices, dense, out in prob.sets:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            prob.eng(slices, dense, out)
+        graphs.append(g)
+    for k in range(warmup):
+        if prob.flush is not None:
+            prob.flush.zero_()
+        graphs[k % prob.n_sets].replay()
+    torch.cuda.synchronize()
+    if dist_ctx is not None:
+        dist_ctx.barrier()
+    if clocks is not None:
+        clocks.start()
+    launches0 = dst.dst_kernel_launches()
+    torch.cuda.synchronize()
+    if prob.flush is None:
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for k in range(steps):
+            graphs[(warmup + k) % prob.n_sets].replay()
+        t1.record()
+        torch.cuda.synchronize()
+        total_ms = t0.elapsed_time(t1)
+    else:
+        ev = []
+        for k in range(steps):
+            prob.flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); graphs[(warmup + k) % prob.n_sets].replay(); b.record()
+            ev.append((a, b))
+        torch.cuda.synchronize()
+        total_ms = float(sum(a.elapsed_time(b) for a, b in ev))
+    clock_info = clocks.stop() if clocks is not None else None
+    if dist_ctx is not None:
+        dist_ctx.barrier()
+    del graphs
+    return total_ms, clock_info
+
+
 def time_e2e(w, device, steps: int, warmup: int):
     """Same metric through the host entry point: pinned host buffers, H2D and D2H inside the timed region."""
     import torch
@@ -271,13 +319,18 @@ def time_oracle(w, max_rows=None, repeats=1):
 
 # ---------------------------------------------------------------------------------------------
 def run_config(name, device, steps, warmup, seed, dist_ctx=None, clocks=None, want_e2e=False, e2e_steps=5,
-               scale=1.0):
+               scale=1.0, use_graph=True):
     import torch
     peak, peak_src = measured_peak()
     w = make_workload(name, seed=seed, scale=scale)
     prob = DeviceProblem(w, device)
-    total_ms, kernel_ms, launches, clock_info = time_device(prob, steps, warmup, dist_ctx, clocks)
+    # eager calls first (per-kernel events, launch count), then the timed steps replayed from CUDA graphs
+    eager_ms, kernel_ms, launches, _ = time_device(prob, steps, warmup, dist_ctx, None)
     res = prob.eng.read_result()
+    if use_graph:
+        total_ms, clock_info = time_device_graph(prob, steps, warmup, dist_ctx, clocks)
+    else:
+        total_ms, _, _, clock_info = time_device(prob, steps, warmup, dist_ctx, clocks)
     ms = total_ms / steps
     kms = float(np.mean(kernel_ms))
     out = {
@@ -285,6 +338,7 @@ def run_config(name, device, steps, warmup, seed, dist_ctx=None, clocks=None, wa
         "frac_of_hbm_peak": prob.balg / ms / 1e6 / peak, "algorithmic_bytes": prob.balg,
         "reduce_kernel_ms": kms, "reduce_kernel_gbs": prob.balg / kms / 1e6,
         "reduce_kernel_frac": prob.balg / kms / 1e6 / peak, "launches": launches, "l2": prob.l2_policy(),
+        "eager_ms_per_step": eager_ms / steps, "cuda_graph": bool(use_graph),
         "n_unique": res["n_unique"], "max_segment": res["max_segment"], "status": res["status"],
         "peak_gbs": peak, "peak_source": peak_src, "clocks": clock_info, "w": w,
     }
@@ -337,6 +391,7 @@ def main():
     ap.add_argument("--headline-only", action="store_true", help="skip the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time eager calls instead of CUDA-graph replays")
     ap.add_argument("--scale", type=float, default=1.0,
                     help="shrink the rows per slice (profiling captures on a small case); 1.0 = the named configuration")
     ap.add_argument("--reference-rows", type=int, default=163840,
@@ -370,7 +425,7 @@ def main():
     seed = replica_seed(args.seed, rank)
     clocks = ClockSampler(local_rank) if rank == 0 else None
     head = run_config(args.workload, device, args.steps, args.warmup, seed, dist_ctx, clocks,
-                      want_e2e=not args.no_e2e, scale=args.scale)
+                      want_e2e=not args.no_e2e, scale=args.scale, use_graph=not args.no_graph)
     w = head.pop("w")
 
     agg = combine_over_ranks(head["ms_per_step"], head["algorithmic_bytes"], w.n_rows_total, dist_ctx, device)
@@ -385,10 +440,10 @@ def main():
         for name in ALL_CONFIGS:
             if name == args.workload:
                 continue
-            r = run_config(name, device, min(args.steps, 200), args.warmup, args.seed)
+            r = run_config(name, device, min(args.steps, 200), args.warmup, args.seed, use_graph=not args.no_graph)
             r.pop("w"); r.pop("clocks")
             others.append({k: r[k] for k in ("workload", "ms_per_step", "gbs", "rows_per_s", "frac_of_hbm_peak",
-                                             "algorithmic_bytes", "reduce_kernel_ms", "reduce_kernel_frac", "l2",
+                                             "algorithmic_bytes", "reduce_kernel_ms", "reduce_kernel_frac", "l2", "eager_ms_per_step",
                                              "n_unique", "max_segment", "status")})
 
     cpu = None
@@ -407,7 +462,10 @@ def main():
             "vs_baseline": None, "dtype": "f32" if w.value_dtype == "f32" else "bf16 in, f32 accumulate",
             "data": "synthetic",
             "config": {"workload": args.workload, "recipe": w.recipe, "vocab": w.vocab, "d": w.d, "R": w.R,
-                       "n_rows_total": w.n_rows_total, "l2": head["l2"], "replicas": world, "scale": args.scale},
+                       "n_rows_total": w.n_rows_total, "l2": head["l2"], "replicas": world, "scale": args.scale,
+                       "timed_as": "CUDA-graph replay of one library call per step" if head["cuda_graph"]
+                       else "eager library calls"},
+            "eager_ms_per_step": head["eager_ms_per_step"],
             "rows_per_s": agg["rows_per_s"], "frac_of_hbm_peak": agg["gbs"] / world / head["peak_gbs"],
             "roofline": {"bound": "hbm", "achieved": head["reduce_kernel_gbs"], "peak": head["peak_gbs"],
                          "unit": "GB/s", "frac": head["reduce_kernel_frac"], "traffic": None,

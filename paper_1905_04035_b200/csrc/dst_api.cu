@@ -75,25 +75,28 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     for (int r = 0; r < R && vector_ok; ++r)
         if (slices[r].n_rows > 0 && !aligned16(slices[r].values)) vector_ok = false;
 
-    if (cudaMemsetAsync(ws, 0, L.zero_bytes, stream) != cudaSuccess) return DST_ERR_CUDA;
-
     const unsigned* perm = pos[L.passes & 1];
-    if (n_total > 0 && n_total <= kSmallMaxRows && vocab <= 65536 && R <= kHistSlices) {
-        // small input: validation, both radix passes and the run lengths in one CTA
-        HistParams P;
-        memset(&P, 0, sizeof P);
-        P.n = R;
+    const bool small = n_total <= kFrontMaxRows && vocab <= 65536 && R <= kHistSlices;
+    if (small) {
+        // small input: one cluster kernel does the whole index side and clears its own tables
+        FrontParams fp;
+        memset(&fp.P, 0, sizeof fp.P);
+        fp.P.n = R;
         int64_t start = 0;
         for (int i = 0; i < R; ++i) {
-            P.s[i] = SliceEntry{slices[i].indices, slices[i].values, (long long)start, (long long)slices[i].n_rows};
+            fp.P.s[i] = SliceEntry{slices[i].indices, slices[i].values, (long long)start, (long long)slices[i].n_rows};
             start += slices[i].n_rows;
         }
-        if (launch_sort_small(P, opts->index_type, hdr, tab, keys[0], pos[0], count, int(n_total), vocab, stream) !=
-            cudaSuccess)
-            return DST_ERR_CUDA;
+        fp.hdr = hdr; fp.tab = tab; fp.perm = pos[0]; fp.offsets = offsets; fp.heavy = heavy;
+        fp.unique_rows = unique_rows; fp.counts_out = counts; fp.result = result; fp.batches = batches;
+        fp.node_cnt = nodecnt; fp.vocab = vocab; fp.n_total = int(n_total); fp.vocab_pad = int(L.vocab_pad);
+        fp.chunk = L.chunk; fp.batch_units = L.batch_units; fp.batch_max = int(L.batch_max);
+        fp.nodecnt_words = int((L.off_batches - L.off_nodecnt) / 4);
+        if (launch_front_cluster(opts->index_type, fp, stream) != cudaSuccess) return DST_ERR_CUDA;
         ++g_launches;
         perm = pos[0];
     } else {
+        if (cudaMemsetAsync(ws, 0, L.zero_bytes, stream) != cudaSuccess) return DST_ERR_CUDA;
         // a1: validate and narrow, at most kHistSlices slices per launch
         int64_t start = 0;
         for (int first = 0; first < R; first += kHistSlices) {
@@ -128,12 +131,12 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
                 return DST_ERR_CUDA;
             ++g_launches;
         }
+        // a3/a5/a6
+        ScanParams sp{hdr, count, offsets, heavy, unique_rows, counts, result, batches,
+                      reinterpret_cast<int*>(ws + L.off_scandesc), int(vocab), int(L.vocab_pad), L.chunk, L.batch_units};
+        if (launch_scan(opts->index_type, sp, stream) != cudaSuccess) return DST_ERR_CUDA;
+        ++g_launches;
     }
-    // a3/a5/a6
-    ScanParams sp{hdr, count, offsets, heavy, unique_rows, counts, result, batches,
-                  reinterpret_cast<int*>(ws + L.off_scandesc), int(vocab), int(L.vocab_pad), L.chunk, L.batch_units};
-    if (launch_scan(opts->index_type, sp, stream) != cudaSuccess) return DST_ERR_CUDA;
-    ++g_launches;
     // a7/a8
     MainArgs a;
     a.hdr = hdr; a.offsets = offsets; a.perm = perm; a.tab = tab; a.heavy = heavy;

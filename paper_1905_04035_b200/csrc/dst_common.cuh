@@ -13,9 +13,9 @@ namespace dst {
 constexpr int kSortThreads = 256;           // threads of the histogram and radix-pass kernels
 constexpr int kSortItems = 16;              // keys per thread of a radix pass
 constexpr int kTile = kSortThreads * kSortItems;  // 4096 keys per CTA
-constexpr int kSmallThreads = 1024;          // the one-CTA sort for small inputs
-constexpr int kSmallGroups = 32;            // groups of 32 entries per warp (at most)
-constexpr int kSmallMaxRows = kSmallThreads * kSmallGroups;   // 32768
+constexpr int kClusterCtas = 8;             // the one-kernel index path for small inputs: CTAs per cluster,
+constexpr int kFrontThreads = 1024;         // threads per CTA,
+constexpr int kFrontMaxRows = 65535;        // largest input (positions are packed into 16 bits)
 constexpr int kPrepItems = 8;               // indices per thread of the validation kernel
 constexpr int kPrepTile = kSortThreads * kPrepItems;
 constexpr int kMaxPasses = 4;               // 8-bit digits, keys below 2^31
@@ -209,8 +209,22 @@ cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeade
 cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
                               unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
                               int pass, int capacity, cudaStream_t stream);
-cudaError_t launch_sort_small(const HistParams& P, int index_type, WsHeader* hdr, SliceEntry* tab, unsigned* skeys,
-                              unsigned* perm, unsigned* count, int n_total, long long vocab, cudaStream_t stream);
+struct FrontParams {
+    HistParams P;
+    WsHeader* hdr;
+    SliceEntry* tab;
+    unsigned* perm;
+    int* offsets;
+    HeavyInfo* heavy;
+    void* unique_rows;
+    int* counts_out;
+    dst_result_t* result;
+    int2* batches;
+    unsigned* node_cnt;
+    long long vocab;
+    int n_total, vocab_pad, chunk, batch_units, batch_max, nodecnt_words;
+};
+cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStream_t stream);
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
                           cudaStream_t stream);
 cudaError_t launch_scan(int index_type, const ScanParams& p, cudaStream_t stream);
@@ -223,6 +237,23 @@ __device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
 __device__ __forceinline__ int warp_id() { return threadIdx.x >> 5; }
 
 __device__ __forceinline__ void raise_status(WsHeader* hdr, int code) { atomicMax(&hdr->status, code); }
+
+// Lanes of the warp whose 8-bit digit equals this lane's, among the lanes with `valid` set
+// (eight ballots; the result is meaningless for lanes without `valid`).
+__device__ __forceinline__ unsigned match_digit(unsigned dg, bool valid) {
+    unsigned m = __ballot_sync(0xFFFFFFFFu, valid);
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+        const bool bit = (dg >> b) & 1u;
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, bit);
+        m &= bit ? bal : ~bal;
+    }
+    return m;
+}
+
+// Units a row contributes to the light work items: its entries and the unit that closes it; a heavy
+// row only keeps its place.
+__host__ __device__ __forceinline__ int row_units(int cc, int chunk) { return cc > chunk ? 1 : cc + 1; }
 
 // Number of combine-tree nodes above the chunk level for a row split into n chunks.
 __host__ __device__ __forceinline__ int upper_nodes(int n) {

@@ -1,0 +1,359 @@
+// Index side of densify for small inputs, in one kernel: a thread-block cluster of kClusterCtas
+// CTAs validates the indices, sorts them (two stable 8-bit radix passes), takes the run lengths and
+// scans them into every table the row-reduction kernel needs.
+//
+// Why a cluster: for a Transformer batch of a few thousand tokens (the paper's Section 3 setting)
+// the index work is pure latency.  Spread over separate kernels it costs more launches than work;
+// in one CTA it is bound by one SM's instruction rate.  Eight CTAs on eight SMs share the work and
+// exchange what they must through distributed shared memory and cluster barriers:
+//   - the per-digit counts of each CTA (to place a CTA's entries behind those of the CTAs before it),
+//   - the entries themselves: pass 0 scatters each packed entry (key << 16 | position) into the
+//     shared memory of the CTA that owns that part of the sorted order,
+//   - count[v], kept in shared memory, a slice of the vocabulary per CTA,
+//   - the per-CTA sums of the final scan.
+// Nothing spins: the only waits are cluster barriers that every thread of every CTA reaches the same
+// number of times.  The kernel also clears the few global tables that must start at zero, so this
+// path needs no memset.
+//
+// Limits: n_total <= kFrontMaxRows (positions fit 16 bits), vocab <= 65536 (keys fit 16 bits),
+// R <= kHistSlices (the slice table travels as a kernel parameter).
+#include <cooperative_groups.h>
+
+#include "dst_common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace dst {
+
+struct FrontArgs {
+    HistParams P;              // the slices
+    WsHeader* hdr;
+    SliceEntry* tab;
+    unsigned* perm;
+    int* offsets;
+    HeavyInfo* heavy;
+    void* unique_rows;
+    int* counts_out;
+    dst_result_t* result;
+    int2* batches;
+    unsigned* node_cnt;
+    long long vocab;
+    int n_total, vocab_pad, chunk, batch_units, batch_max, nodecnt_words;
+    int lw;                    // entries per warp (multiple of 32); a CTA's slice of the sorted order holds 32 * lw
+    int rpt;                   // vocabulary rows per thread in the scan; a CTA's slice of count[] holds 1024 * rpt
+};
+
+constexpr int kFrontWarps = kFrontThreads / 32;
+constexpr int kFrontGroups = 8;       // groups of 32 entries per warp, at most (kFrontMaxRows / 256 / 32)
+constexpr int kFrontRpt = 8;          // rows per thread, at most (65536 / 8192)
+
+// one group of 32 entries: add it to the warp's running digit counters and return this lane's
+// rank among the warp's entries so far with the same digit (wh: this warp's 256 counters)
+__device__ __forceinline__ unsigned rank_step(unsigned short* wh, bool valid, unsigned dg, int lane) {
+    const unsigned m = match_digit(dg & 255u, valid);
+    const int leader = valid ? __ffs(m) - 1 : lane;
+    unsigned pre = 0;
+    if (valid && lane == leader) { pre = wh[dg]; wh[dg] = (unsigned short)(pre + __popc(m)); }
+    pre = __shfl_sync(0xFFFFFFFFu, pre, leader);
+    __syncwarp();
+    return pre + __popc(m & ((1u << lane) - 1u));
+}
+
+// After every warp has counted its digits into wh[w][d]: turn the counts into the sorted position
+// of the first entry of (digit d, this CTA, warp w).  One cluster barrier inside.  Returns the
+// number of entries over the whole cluster.
+__device__ __forceinline__ unsigned cluster_bases(cg::cluster_group& cluster, unsigned short (*wh)[256],
+                                                  unsigned* cta_tot, unsigned* s_warp_tot, unsigned* s_total) {
+    const int lane = lane_id(), warp = warp_id();
+    const unsigned rank = cluster.block_rank();
+    unsigned tot = 0;
+    if (threadIdx.x < 256) {
+#pragma unroll 8
+        for (int w = 0; w < kFrontWarps; ++w) { unsigned t = wh[w][threadIdx.x]; wh[w][threadIdx.x] = (unsigned short)tot; tot += t; }
+        cta_tot[threadIdx.x] = tot;
+    }
+    cluster.sync();                                   // every CTA's per-digit totals are in place
+    unsigned before = 0, all = 0;
+    if (threadIdx.x < 256) {
+#pragma unroll
+        for (unsigned c = 0; c < (unsigned)kClusterCtas; ++c) {
+            const unsigned t = cluster.map_shared_rank(cta_tot, c)[threadIdx.x];
+            if (c < rank) before += t;
+            all += t;
+        }
+    }
+    unsigned inc = all;                               // exclusive scan of the digit totals over the 256 digits
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { unsigned t = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t; }
+    if (lane == 31 && warp < 8) s_warp_tot[warp] = inc;
+    __syncthreads();
+    if (threadIdx.x < 256) {
+        unsigned base = inc - all + before;
+        for (int w = 0; w < warp; ++w) base += s_warp_tot[w];
+#pragma unroll 8
+        for (int w = 0; w < kFrontWarps; ++w) wh[w][threadIdx.x] = (unsigned short)(wh[w][threadIdx.x] + base);
+        if (threadIdx.x == 255) *s_total = base - before + all;
+    }
+    __syncthreads();
+    return *s_total;
+}
+
+struct Sum6 { int v[6]; };   // 0 offset, 1 unique, 2 heavy rows, 3 chunks, 4 upper nodes, 5 units of the light work items
+
+template <typename IT>
+__global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kFrontThreads, 1)
+k_front_cluster(const __grid_constant__ FrontArgs f) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ unsigned short wh[kFrontWarps][256];
+    __shared__ unsigned cta_tot[256];
+    __shared__ unsigned s_warp_tot[8];
+    __shared__ unsigned s_total;
+    __shared__ int s_scan[kFrontWarps][6];
+    __shared__ int cta_sum[6];
+    __shared__ int s_maxseg[kFrontWarps];
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int lane = lane_id(), warp = warp_id();
+    const int S = 32 * f.lw;                         // entries of the sorted order this CTA owns
+    const int Vs = kFrontThreads * f.rpt;            // rows of count[] this CTA owns
+    unsigned* packed = reinterpret_cast<unsigned*>(dyn);                          // [S] key << 16 | position
+    unsigned* cnt = packed + S;                                                   // [Vs]
+    unsigned short* skey = reinterpret_cast<unsigned short*>(cnt + Vs);           // [S] sorted keys
+    WsHeader* hdr = f.hdr;
+    const int gt = rank * kFrontThreads + threadIdx.x;   // thread id in the cluster
+    constexpr int kAllThreads = kClusterCtas * kFrontThreads;
+
+    // ---- clear what must start at zero
+    for (int i = threadIdx.x; i < Vs; i += kFrontThreads) cnt[i] = 0;
+    for (int i = gt; i < f.batch_max; i += kAllThreads) f.batches[i] = make_int2(0, 0);
+    for (int i = gt; i < f.nodecnt_words; i += kAllThreads) f.node_cnt[i] = 0;
+    if (rank == 0) {
+        if (threadIdx.x < (int)(sizeof(WsHeader) / 4)) reinterpret_cast<unsigned*>(hdr)[threadIdx.x] = 0;
+        if (threadIdx.x < f.P.n) f.tab[threadIdx.x] = f.P.s[threadIdx.x];
+    }
+    for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(wh[warp])[s] = 0;
+
+    // ---- a1: load and validate.  Warp gw of the cluster owns entries [gw * lw, gw * lw + lw).
+    const int gw = rank * kFrontWarps + warp;
+    const int ng = f.lw / 32;
+    unsigned key[kFrontGroups];
+    {
+        int r = 0;
+#pragma unroll
+        for (int g = 0; g < kFrontGroups; ++g) {
+            key[g] = kInvalidKey;
+            const int e = gw * f.lw + g * 32 + lane;
+            if (g < ng && e < f.n_total) {
+                while (r + 1 < f.P.n && (long long)e >= f.P.s[r + 1].start) ++r;
+                const long long v = (long long)static_cast<const IT*>(f.P.s[r].indices)[(long long)e - f.P.s[r].start];
+                if (v >= 0 && v < f.vocab) key[g] = (unsigned)v;
+            }
+        }
+    }
+    __syncwarp();
+    // ---- a4, pass 0: low digit; registers -> the shared memory of the CTA that owns the target position
+#pragma unroll
+    for (int g = 0; g < kFrontGroups; ++g)
+        if (g < ng) rank_step(wh[warp], key[g] != kInvalidKey, key[g] & 255u, lane);
+    __syncthreads();
+    const int n_valid = (int)cluster_bases(cluster, wh, cta_tot, s_warp_tot, &s_total);
+#pragma unroll
+    for (int g = 0; g < kFrontGroups; ++g) {
+        if (g < ng) {
+            const bool valid = key[g] != kInvalidKey;
+            const unsigned q = rank_step(wh[warp], valid, key[g] & 255u, lane);
+            if (valid) {
+                const unsigned owner = q / (unsigned)S;
+                cluster.map_shared_rank(packed, owner)[q - owner * (unsigned)S] =
+                    (key[g] << 16) | (unsigned)(gw * f.lw + g * 32 + lane);
+            }
+        }
+    }
+    for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(wh[warp])[s] = 0;
+    cluster.sync();                                   // all of pass 0 has landed
+    // ---- pass 1: high digit; this CTA's slice [rank * S, rank * S + S) -> perm (global) and skey (owner's shared memory)
+    for (int g = 0; g < ng; ++g) {
+        const int e = warp * f.lw + g * 32 + lane;
+        const bool valid = rank * S + e < n_valid;
+        const unsigned x = valid ? packed[e] : 0u;
+        rank_step(wh[warp], valid, x >> 24, lane);
+    }
+    __syncthreads();
+    cluster_bases(cluster, wh, cta_tot, s_warp_tot, &s_total);
+    for (int g = 0; g < ng; ++g) {
+        const int e = warp * f.lw + g * 32 + lane;
+        const bool valid = rank * S + e < n_valid;
+        const unsigned x = valid ? packed[e] : 0u;
+        const unsigned q = rank_step(wh[warp], valid, x >> 24, lane);
+        if (valid) {
+            f.perm[q] = x & 0xFFFFu;
+            const unsigned owner = q / (unsigned)S;
+            cluster.map_shared_rank(skey, owner)[q - owner * (unsigned)S] = (unsigned short)(x >> 16);
+        }
+    }
+    cluster.sync();                                   // the sorted keys are in place
+    // ---- a2: run lengths.  The first entry of a run subtracts its position from count[key], the last
+    // adds its position + 1; count[] lives in shared memory, rows [c * Vs, c * Vs + Vs) in CTA c.
+    for (int e = threadIdx.x; e < S; e += kFrontThreads) {
+        const int i = rank * S + e;
+        if (i < n_valid) {
+            const unsigned k = skey[e];
+            unsigned prev = ~k, next = ~k;
+            if (i > 0) prev = e > 0 ? skey[e - 1] : cluster.map_shared_rank(skey, rank - 1)[S - 1];
+            if (i + 1 < n_valid) next = e + 1 < S ? skey[e + 1] : cluster.map_shared_rank(skey, rank + 1)[0];
+            const unsigned owner = k / (unsigned)Vs;
+            unsigned* c = cluster.map_shared_rank(cnt, owner) + (k - owner * (unsigned)Vs);
+            if (prev != k) atomicSub(c, (unsigned)i);
+            if (next != k) atomicAdd(c, (unsigned)i + 1u);
+        }
+    }
+    cluster.sync();                                   // count[] is complete
+    // ---- a3 + a5 + a6: scan of count[].  Thread t of CTA c owns rows c * Vs + t * rpt + [0, rpt).
+    IT* unique_rows = static_cast<IT*>(f.unique_rows);
+    const int chunk = f.chunk, B = f.batch_units, vocab = (int)f.vocab;
+    const int l0 = threadIdx.x * f.rpt;              // first owned row, local
+    const int e0 = rank * Vs + l0;                   // ... and global
+    int c[kFrontRpt];
+    Sum6 mine{};
+    int maxseg = 0;
+#pragma unroll
+    for (int q = 0; q < kFrontRpt; ++q) {
+        c[q] = q < f.rpt ? (int)cnt[l0 + q] : 0;
+        const int cc = c[q];
+        mine.v[0] += cc;
+        mine.v[1] += cc > 0;
+        if (q < f.rpt && e0 + q < vocab) mine.v[5] += row_units(cc, chunk);
+        if (cc > chunk) {
+            const int n = (cc + chunk - 1) / chunk;
+            mine.v[2] += 1; mine.v[3] += n; mine.v[4] += upper_nodes(n);
+        }
+        maxseg = max(maxseg, cc);
+    }
+    int prev_cost = 0;                               // units of the row before this thread's first one
+    if (e0 > 0 && e0 < f.vocab_pad) {
+        const unsigned pc = l0 > 0 ? cnt[l0 - 1] : cluster.map_shared_rank(cnt, rank - 1)[Vs - 1];
+        prev_cost = row_units((int)pc, chunk);
+    }
+    Sum6 inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+        for (int q = 0; q < 6; ++q) {
+            int t = __shfl_up_sync(0xFFFFFFFFu, inc.v[q], o);
+            if (lane >= o) inc.v[q] += t;
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) maxseg = max(maxseg, __shfl_down_sync(0xFFFFFFFFu, maxseg, o));
+    if (lane == 31) {
+#pragma unroll
+        for (int q = 0; q < 6; ++q) s_scan[warp][q] = inc.v[q];
+    }
+    if (lane == 0) s_maxseg[warp] = maxseg;
+    __syncthreads();
+    Sum6 run, total;
+#pragma unroll
+    for (int q = 0; q < 6; ++q) {
+        int before = 0, all = 0;
+        for (int w = 0; w < kFrontWarps; ++w) { const int t = s_scan[w][q]; if (w < warp) before += t; all += t; }
+        run.v[q] = inc.v[q] - mine.v[q] + before;
+        total.v[q] = all;
+    }
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int q = 0; q < 6; ++q) cta_sum[q] = total.v[q];
+        int m = 0;
+        for (int w = 0; w < kFrontWarps; ++w) m = max(m, s_maxseg[w]);
+        if (m > 0) atomicMax(&hdr->max_segment, m);
+    }
+    cluster.sync();                                   // every CTA's sums are in place
+    Sum6 grand{};
+#pragma unroll
+    for (int q = 0; q < 6; ++q) {
+        for (int cc = 0; cc < kClusterCtas; ++cc) {
+            const int t = cluster.map_shared_rank(cta_sum, cc)[q];
+            if (cc < rank) run.v[q] += t;
+            grand.v[q] += t;
+        }
+    }
+    if (e0 < f.vocab_pad) {
+        int rem = run.v[5] % B;                      // units before row e0, modulo the batch size
+        int b = run.v[5] / B;
+#pragma unroll
+        for (int q = 0; q < kFrontRpt; ++q) {
+            const int v = e0 + q;
+            if (q < f.rpt && v < f.vocab_pad) {
+                const int cc = c[q];
+                f.offsets[v] = run.v[0];
+                if (cc > 0) {
+                    if (unique_rows) unique_rows[run.v[1]] = (IT)v;
+                    if (f.counts_out) f.counts_out[run.v[1]] = cc;
+                    run.v[1] += 1;
+                }
+                if (cc > chunk) {
+                    // a6: a heavy row becomes n chunk items and a combine tree
+                    const int n = (cc + chunk - 1) / chunk;
+                    f.heavy[run.v[2]] = HeavyInfo{v, run.v[3], run.v[4], n, run.v[0], cc, {0, 0}};
+                    run.v[2] += 1; run.v[3] += n; run.v[4] += upper_nodes(n);
+                }
+                run.v[0] += cc;
+                if (v < vocab) {
+                    // light work items: row v belongs to batch floor(units before v / batch size)
+                    const int cost = row_units(cc, chunk);
+                    if (v == 0 || prev_cost > rem) f.batches[b].x = v + 1;
+                    rem += cost;
+                    if (v == vocab - 1 || rem >= B) f.batches[b].y = v + 1;
+                    if (rem >= B) { b += rem / B; rem %= B; }
+                    prev_cost = cost;
+                }
+            }
+        }
+    }
+    cluster.sync();       // all tables and the header's max_segment are written; nobody reads a peer's shared memory after this
+    if (rank == 0 && threadIdx.x == 0) {
+        f.offsets[f.vocab_pad] = grand.v[0];
+        hdr->n_valid = grand.v[0];
+        hdr->n_unique = grand.v[1];
+        hdr->n_heavy = grand.v[2];
+        hdr->n_chunks = grand.v[3];
+        hdr->n_upper = grand.v[4];
+        hdr->n_batches = grand.v[5] > 0 ? (grand.v[5] - 1) / B + 1 : 0;
+        const long long bad = (long long)f.n_total - n_valid;
+        hdr->n_bad = (unsigned long long)bad;
+        if (bad) raise_status(hdr, DST_ERR_INDEX_OUT_OF_RANGE);
+        if (f.result) {
+            f.result->n_unique = grand.v[1];
+            f.result->n_out_of_range = bad;
+            f.result->max_segment = *reinterpret_cast<volatile int*>(&hdr->max_segment);
+        }
+    }
+}
+
+cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStream_t stream) {
+    FrontArgs f;
+    f.P = p.P; f.hdr = p.hdr; f.tab = p.tab; f.perm = p.perm; f.offsets = p.offsets; f.heavy = p.heavy;
+    f.unique_rows = p.unique_rows; f.counts_out = p.counts_out; f.result = p.result; f.batches = p.batches;
+    f.node_cnt = p.node_cnt; f.vocab = p.vocab; f.n_total = p.n_total; f.vocab_pad = p.vocab_pad; f.chunk = p.chunk;
+    f.batch_units = p.batch_units; f.batch_max = p.batch_max; f.nodecnt_words = p.nodecnt_words;
+    const int per_warp = (p.n_total + kClusterCtas * kFrontWarps - 1) / (kClusterCtas * kFrontWarps);
+    f.lw = (per_warp + 31) / 32 * 32;
+    if (f.lw < 32) f.lw = 32;
+    f.rpt = (p.vocab_pad + kClusterCtas * kFrontThreads - 1) / (kClusterCtas * kFrontThreads);
+    if (f.rpt < 1) f.rpt = 1;
+    if (f.lw > 32 * kFrontGroups || f.rpt > kFrontRpt) return cudaErrorInvalidValue;
+    const size_t S = size_t(32) * f.lw, Vs = size_t(kFrontThreads) * f.rpt;
+    const size_t smem = S * 4 + Vs * 4 + S * 2;
+    cudaError_t e;
+    if (index_type == DST_I64) {
+        e = cudaFuncSetAttribute(k_front_cluster<long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_front_cluster<long long><<<kClusterCtas, kFrontThreads, smem, stream>>>(f);
+    } else {
+        e = cudaFuncSetAttribute(k_front_cluster<int>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_front_cluster<int><<<kClusterCtas, kFrontThreads, smem, stream>>>(f);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace dst

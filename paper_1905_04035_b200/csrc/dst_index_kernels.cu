@@ -11,7 +11,7 @@
 //   k_radix_pass  one per 8-bit digit, least significant first, stable
 //   k_bounds      run lengths of the sorted keys -> count[v]
 //   k_scan        count[] -> offsets, unique rows, heavy-row chunks, row batches
-// Small inputs take k_front_small, which does all of it in one CTA.
+// Small inputs take k_front_cluster (dst_front_cluster.cu), which does all of it in one kernel.
 #include "dst_common.cuh"
 
 namespace dst {
@@ -49,8 +49,8 @@ k_prep(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, unsigne
         bad += in && !ok;
         // equal digits inside the warp are added once (frequent rows would otherwise serialise)
         for (int p = 0; p < passes; ++p) {
-            const unsigned dg = ok ? ((key >> (8 * p)) & 255u) : (0x10000u | lane);
-            const unsigned m = __match_any_sync(0xFFFFFFFFu, dg);
+            const unsigned dg = (key >> (8 * p)) & 255u;
+            const unsigned m = match_digit(dg, ok);
             if (ok && lane == __ffs(m) - 1) atomicAdd(&dh[p * 256 + dg], (unsigned)__popc(m));
         }
     }
@@ -137,9 +137,9 @@ k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, c
 #pragma unroll
     for (int k = 0; k < kSortItems; ++k) {
         const bool valid = key[k] != kInvalidKey;
-        unsigned dg = valid ? ((key[k] >> shift) & 255u) : (0x10000u | lane);
-        unsigned m = __match_any_sync(0xFFFFFFFFu, dg);
-        int leader = __ffs(m) - 1;
+        unsigned dg = (key[k] >> shift) & 255u;
+        unsigned m = match_digit(dg, valid);
+        int leader = valid ? __ffs(m) - 1 : lane;
         unsigned pre = 0;
         if (valid && lane == leader) { pre = wh[warp][dg]; wh[warp][dg] = pre + __popc(m); }
         pre = __shfl_sync(0xFFFFFFFFu, pre, leader);
@@ -219,7 +219,6 @@ struct ScanArgs {
 };
 
 
-__device__ __forceinline__ int row_units(int cc, int chunk) { return cc > chunk ? 1 : cc + 1; }
 
 // exclusive scan over the CTA (kScanThreads threads) of six counters at once
 __device__ __forceinline__ Scan6 block_exclusive_scan(Scan6 x, Scan6& total, int (*sm)[6]) {
@@ -419,133 +418,6 @@ k_scan(const ScanArgs s) {
     }
 }
 
-// ---------------------------------------------------------------------------
-// Small inputs: a1 + a4 + a2 in one CTA.  The keys stay on chip between the two radix passes
-// (registers, then one packed word per entry in shared memory), so there is no look-back and no
-// intermediate global traffic.  Needs n_total <= kSmallMaxRows, vocab <= 65536, R <= kHistSlices.
-//
-// Warp w owns the entries [w * L, (w + 1) * L) in input order and walks them 32 at a time, so
-// ranking inside a warp by lane order and across warps by warp order is stable.
-// ---------------------------------------------------------------------------
-struct SmallRank {
-    // one group of 32 entries: add the group to the warp's running digit counters and return
-    // this lane's rank among the entries of the tile with the same digit (wh: this warp's row)
-    static __device__ __forceinline__ unsigned step(unsigned short* wh, bool valid, unsigned dg, int lane) {
-        const unsigned m = __match_any_sync(0xFFFFFFFFu, valid ? dg : (0x10000u | lane));
-        const int leader = __ffs(m) - 1;
-        unsigned pre = 0;
-        if (valid && lane == leader) { pre = wh[dg]; wh[dg] = (unsigned short)(pre + __popc(m)); }
-        pre = __shfl_sync(0xFFFFFFFFu, pre, leader);
-        __syncwarp();
-        return pre + __popc(m & ((1u << lane) - 1u));
-    }
-};
-
-// wh[w][d] holds per-warp digit counts: turn them into the position of the first entry of
-// (digit d, warp w) in the sorted order; returns the number of entries (valid at thread 255)
-__device__ __forceinline__ unsigned small_bases(unsigned short (*wh)[256], unsigned* s_warp_tot) {
-    const int lane = lane_id(), warp = warp_id();
-    unsigned tot = 0;
-    if (threadIdx.x < 256) {
-#pragma unroll 8
-        for (int w = 0; w < kSmallThreads / 32; ++w) { unsigned t = wh[w][threadIdx.x]; wh[w][threadIdx.x] = (unsigned short)tot; tot += t; }
-    }
-    unsigned inc = tot;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { unsigned t = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t; }
-    if (lane == 31 && warp < 8) s_warp_tot[warp] = inc;
-    __syncthreads();
-    unsigned n_all = 0;
-    if (threadIdx.x < 256) {
-        unsigned base = inc - tot;
-        for (int w = 0; w < warp; ++w) base += s_warp_tot[w];
-#pragma unroll 8
-        for (int w = 0; w < kSmallThreads / 32; ++w) wh[w][threadIdx.x] = (unsigned short)(wh[w][threadIdx.x] + base);
-        n_all = base + tot;
-    }
-    __syncthreads();
-    return n_all;
-}
-
-template <typename IT>
-__global__ void __launch_bounds__(kSmallThreads)
-k_sort_small(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, SliceEntry* __restrict__ tab,
-             unsigned* __restrict__ skeys, unsigned* __restrict__ perm, unsigned* __restrict__ count, int n_total,
-             long long vocab) {
-    extern __shared__ unsigned packed[];             // pass 0 output: key << 16 | position
-    __shared__ unsigned short wh[kSmallThreads / 32][256];
-    __shared__ unsigned s_warp_tot[8];
-    __shared__ int s_nvalid;
-    const int lane = lane_id(), warp = warp_id();
-    if (threadIdx.x < P.n) tab[P.first + threadIdx.x] = P.s[threadIdx.x];
-    for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(wh[warp])[s] = 0;
-
-    // ---- load and validate: warp `warp` owns entries [warp * L, warp * L + L)
-    const int L = ((n_total + kSmallThreads - 1) / kSmallThreads) * 32;
-    const int ng = L / 32;                           // groups per warp, <= kSmallGroups
-    unsigned key[kSmallGroups];
-    {
-        int r = 0;
-#pragma unroll
-        for (int g = 0; g < kSmallGroups; ++g) {
-            key[g] = kInvalidKey;
-            const int e = warp * L + g * 32 + lane;
-            if (g < ng && e < n_total) {
-                while (r + 1 < P.n && (long long)e >= P.s[r + 1].start) ++r;
-                const long long v = (long long)static_cast<const IT*>(P.s[r].indices)[(long long)e - P.s[r].start];
-                if (v >= 0 && v < vocab) key[g] = (unsigned)v;
-            }
-        }
-    }
-    __syncwarp();
-    // ---- pass 0: low digit, registers -> shared
-#pragma unroll
-    for (int g = 0; g < kSmallGroups; ++g)
-        if (g < ng) SmallRank::step(wh[warp], key[g] != kInvalidKey, key[g] & 255u, lane);
-    __syncthreads();
-    const unsigned n_all = small_bases(wh, s_warp_tot);
-    if (threadIdx.x == 255) s_nvalid = (int)n_all;
-#pragma unroll
-    for (int g = 0; g < kSmallGroups; ++g) {
-        if (g < ng) {
-            const bool valid = key[g] != kInvalidKey;
-            const unsigned q = SmallRank::step(wh[warp], valid, key[g] & 255u, lane);
-            if (valid) packed[q] = (key[g] << 16) | (unsigned)(warp * L + g * 32 + lane);
-        }
-    }
-    __syncthreads();
-    const int n_valid = s_nvalid;
-    // ---- pass 1: high digit, shared -> global
-    for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(wh[warp])[s] = 0;
-    __syncwarp();
-    const int L1 = ((n_valid + kSmallThreads - 1) / kSmallThreads) * 32;
-    for (int g = 0; g < L1 / 32; ++g) {
-        const int e = warp * L1 + g * 32 + lane;
-        const bool valid = e < n_valid;
-        const unsigned x = valid ? packed[e] : 0u;
-        SmallRank::step(wh[warp], valid, x >> 24, lane);
-    }
-    __syncthreads();
-    small_bases(wh, s_warp_tot);
-    for (int g = 0; g < L1 / 32; ++g) {
-        const int e = warp * L1 + g * 32 + lane;
-        const bool valid = e < n_valid;
-        const unsigned x = valid ? packed[e] : 0u;
-        const unsigned q = SmallRank::step(wh[warp], valid, x >> 24, lane);
-        if (valid) { perm[q] = x & 0xFFFFu; skeys[q] = x >> 16; }
-    }
-    __syncthreads();
-    // ---- a2: run lengths of the sorted keys (see k_bounds)
-    for (int i = threadIdx.x; i < n_valid; i += kSmallThreads) {
-        const unsigned k = skeys[i];
-        const unsigned prev = i > 0 ? skeys[i - 1] : ~k;
-        const unsigned next = i + 1 < n_valid ? skeys[i + 1] : ~k;
-        if (prev != k) atomicSub(&count[k], (unsigned)i);
-        if (next != k) atomicAdd(&count[k], (unsigned)i + 1u);
-    }
-    if (threadIdx.x == 0) hdr->n_bad = (unsigned long long)(n_total - n_valid);
-}
-
 // ---- host-side launchers ------------------------------------------------------
 cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeader* hdr, unsigned* digit_hist,
                         unsigned* keys, SliceEntry* tab, long long vocab, int passes, cudaStream_t stream) {
@@ -562,22 +434,6 @@ cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_key
                               int pass, int capacity, cudaStream_t stream) {
     k_radix_pass<<<n_tiles, kSortThreads, 0, stream>>>(hdr, in_keys, in_pos, out_keys, out_pos, digit_hist, desc,
                                                        pass, capacity);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_sort_small(const HistParams& P, int index_type, WsHeader* hdr, SliceEntry* tab, unsigned* skeys,
-                              unsigned* perm, unsigned* count, int n_total, long long vocab, cudaStream_t stream) {
-    const size_t smem = size_t(n_total) * 4;
-    cudaError_t e;
-    if (index_type == DST_I64) {
-        e = cudaFuncSetAttribute(k_sort_small<long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmallMaxRows * 4);
-        if (e != cudaSuccess) return e;
-        k_sort_small<long long><<<1, kSmallThreads, smem, stream>>>(P, hdr, tab, skeys, perm, count, n_total, vocab);
-    } else {
-        e = cudaFuncSetAttribute(k_sort_small<int>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmallMaxRows * 4);
-        if (e != cudaSuccess) return e;
-        k_sort_small<int><<<1, kSmallThreads, smem, stream>>>(P, hdr, tab, skeys, perm, count, n_total, vocab);
-    }
     return cudaGetLastError();
 }
 
