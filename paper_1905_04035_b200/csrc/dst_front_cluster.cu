@@ -110,6 +110,7 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
     __shared__ unsigned s_total;
     __shared__ int s_scan[kFrontWarps][6];
     __shared__ int cta_sum[6];
+    __shared__ int s_before[6], s_grand[6];
     __shared__ int s_maxseg[kFrontWarps];
 
     cg::cluster_group cluster = cg::this_cluster();
@@ -152,41 +153,48 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
         }
     }
     __syncwarp();
-    // ---- a4, pass 0: low digit; registers -> the shared memory of the CTA that owns the target position
+    // ---- a4, pass 0: low digit; registers -> the shared memory of the CTA that owns the target position.
+    // rk[g] is the entry's rank among the warp's entries with the same digit; once the counters have
+    // become positions (cluster_bases) the target is wh[warp][digit] + rk[g].
+    unsigned short rk[kFrontGroups];
 #pragma unroll
-    for (int g = 0; g < kFrontGroups; ++g)
-        if (g < ng) rank_step(wh[warp], key[g] != kInvalidKey, key[g] & 255u, lane);
+    for (int g = 0; g < kFrontGroups; ++g) {
+        rk[g] = 0;
+        if (g < ng) rk[g] = (unsigned short)rank_step(wh[warp], key[g] != kInvalidKey, key[g] & 255u, lane);
+    }
     __syncthreads();
     const int n_valid = (int)cluster_bases(cluster, wh, cta_tot, s_warp_tot, &s_total);
 #pragma unroll
     for (int g = 0; g < kFrontGroups; ++g) {
-        if (g < ng) {
-            const bool valid = key[g] != kInvalidKey;
-            const unsigned q = rank_step(wh[warp], valid, key[g] & 255u, lane);
-            if (valid) {
-                const unsigned owner = q / (unsigned)S;
-                cluster.map_shared_rank(packed, owner)[q - owner * (unsigned)S] =
-                    (key[g] << 16) | (unsigned)(gw * f.lw + g * 32 + lane);
-            }
+        if (g < ng && key[g] != kInvalidKey) {
+            const unsigned q = (unsigned)wh[warp][key[g] & 255u] + rk[g];
+            const unsigned owner = q / (unsigned)S;
+            cluster.map_shared_rank(packed, owner)[q - owner * (unsigned)S] =
+                (key[g] << 16) | (unsigned)(gw * f.lw + g * 32 + lane);
         }
     }
+    __syncthreads();                                  // every warp has read its positions
     for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(wh[warp])[s] = 0;
     cluster.sync();                                   // all of pass 0 has landed
     // ---- pass 1: high digit; this CTA's slice [rank * S, rank * S + S) -> perm (global) and skey (owner's shared memory)
-    for (int g = 0; g < ng; ++g) {
+#pragma unroll
+    for (int g = 0; g < kFrontGroups; ++g) {
+        key[g] = kInvalidKey; rk[g] = 0;
         const int e = warp * f.lw + g * 32 + lane;
-        const bool valid = rank * S + e < n_valid;
-        const unsigned x = valid ? packed[e] : 0u;
-        rank_step(wh[warp], valid, x >> 24, lane);
+        if (g < ng) {
+            const bool valid = rank * S + e < n_valid;
+            const unsigned x = valid ? packed[e] : 0u;   // a packed entry (never 0xFFFFFFFF: positions stay below 65535)
+            rk[g] = (unsigned short)rank_step(wh[warp], valid, x >> 24, lane);
+            if (valid) key[g] = x;
+        }
     }
     __syncthreads();
     cluster_bases(cluster, wh, cta_tot, s_warp_tot, &s_total);
-    for (int g = 0; g < ng; ++g) {
-        const int e = warp * f.lw + g * 32 + lane;
-        const bool valid = rank * S + e < n_valid;
-        const unsigned x = valid ? packed[e] : 0u;
-        const unsigned q = rank_step(wh[warp], valid, x >> 24, lane);
-        if (valid) {
+#pragma unroll
+    for (int g = 0; g < kFrontGroups; ++g) {
+        if (g < ng && key[g] != kInvalidKey) {
+            const unsigned x = key[g];
+            const unsigned q = (unsigned)wh[warp][x >> 24] + rk[g];
             f.perm[q] = x & 0xFFFFu;
             const unsigned owner = q / (unsigned)S;
             cluster.map_shared_rank(skey, owner)[q - owner * (unsigned)S] = (unsigned short)(x >> 16);
@@ -251,31 +259,46 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
     }
     if (lane == 0) s_maxseg[warp] = maxseg;
     __syncthreads();
-    Sum6 run, total;
+    if (warp == 0) {
+        // lane w holds warp w's sums: scan them, leave each warp's exclusive prefix and the CTA's sums
+        Sum6 ws, wi;
 #pragma unroll
-    for (int q = 0; q < 6; ++q) {
-        int before = 0, all = 0;
-        for (int w = 0; w < kFrontWarps; ++w) { const int t = s_scan[w][q]; if (w < warp) before += t; all += t; }
-        run.v[q] = inc.v[q] - mine.v[q] + before;
-        total.v[q] = all;
-    }
-    if (threadIdx.x == 0) {
+        for (int q = 0; q < 6; ++q) { ws.v[q] = s_scan[lane][q]; wi.v[q] = ws.v[q]; }
 #pragma unroll
-        for (int q = 0; q < 6; ++q) cta_sum[q] = total.v[q];
-        int m = 0;
-        for (int w = 0; w < kFrontWarps; ++w) m = max(m, s_maxseg[w]);
-        if (m > 0) atomicMax(&hdr->max_segment, m);
-    }
-    cluster.sync();                                   // every CTA's sums are in place
-    Sum6 grand{};
+        for (int o = 1; o < 32; o <<= 1) {
 #pragma unroll
-    for (int q = 0; q < 6; ++q) {
-        for (int cc = 0; cc < kClusterCtas; ++cc) {
-            const int t = cluster.map_shared_rank(cta_sum, cc)[q];
-            if (cc < rank) run.v[q] += t;
-            grand.v[q] += t;
+            for (int q = 0; q < 6; ++q) {
+                int t = __shfl_up_sync(0xFFFFFFFFu, wi.v[q], o);
+                if (lane >= o) wi.v[q] += t;
+            }
         }
+#pragma unroll
+        for (int q = 0; q < 6; ++q) {
+            s_scan[lane][q] = wi.v[q] - ws.v[q];
+            if (lane == 31) cta_sum[q] = wi.v[q];
+        }
+        int m = s_maxseg[lane];
+        for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_down_sync(0xFFFFFFFFu, m, o));
+        if (lane == 0 && m > 0) atomicMax(&hdr->max_segment, m);
     }
+    __syncthreads();
+    Sum6 run;
+#pragma unroll
+    for (int q = 0; q < 6; ++q) run.v[q] = inc.v[q] - mine.v[q] + s_scan[warp][q];
+    cluster.sync();                                   // every CTA's sums are in place
+    if (threadIdx.x < 6) {
+        int before = 0, all = 0;
+        for (int cc = 0; cc < kClusterCtas; ++cc) {
+            const int t = cluster.map_shared_rank(cta_sum, cc)[threadIdx.x];
+            if (cc < rank) before += t;
+            all += t;
+        }
+        s_before[threadIdx.x] = before;
+        s_grand[threadIdx.x] = all;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 6; ++q) run.v[q] += s_before[q];
     if (e0 < f.vocab_pad) {
         int rem = run.v[5] % B;                      // units before row e0, modulo the batch size
         int b = run.v[5] / B;
@@ -311,18 +334,18 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
     }
     cluster.sync();       // all tables and the header's max_segment are written; nobody reads a peer's shared memory after this
     if (rank == 0 && threadIdx.x == 0) {
-        f.offsets[f.vocab_pad] = grand.v[0];
-        hdr->n_valid = grand.v[0];
-        hdr->n_unique = grand.v[1];
-        hdr->n_heavy = grand.v[2];
-        hdr->n_chunks = grand.v[3];
-        hdr->n_upper = grand.v[4];
-        hdr->n_batches = grand.v[5] > 0 ? (grand.v[5] - 1) / B + 1 : 0;
+        f.offsets[f.vocab_pad] = s_grand[0];
+        hdr->n_valid = s_grand[0];
+        hdr->n_unique = s_grand[1];
+        hdr->n_heavy = s_grand[2];
+        hdr->n_chunks = s_grand[3];
+        hdr->n_upper = s_grand[4];
+        hdr->n_batches = s_grand[5] > 0 ? (s_grand[5] - 1) / B + 1 : 0;
         const long long bad = (long long)f.n_total - n_valid;
         hdr->n_bad = (unsigned long long)bad;
         if (bad) raise_status(hdr, DST_ERR_INDEX_OUT_OF_RANGE);
         if (f.result) {
-            f.result->n_unique = grand.v[1];
+            f.result->n_unique = s_grand[1];
             f.result->n_out_of_range = bad;
             f.result->max_segment = *reinterpret_cast<volatile int*>(&hdr->max_segment);
         }

@@ -444,16 +444,19 @@ struct WarpPipe {
         const unsigned n_chunks = (unsigned)a.hdr->n_chunks;
         const unsigned n_base = n_chunks + (unsigned)a.hdr->n_batches;
         const unsigned n_items = n_base * (unsigned)a.ncb;
+        // The first item of a warp is its own number (no traffic on the shared counter while the whole
+        // grid starts up); later ones come from the counter, fetched one item ahead.
+        const unsigned n_warps = gridDim.x * (unsigned)kPipeWarps;
+        unsigned item = blockIdx.x * (unsigned)kPipeWarps + (unsigned)warp_id();
         bool ok = true;
         unsigned pending = 0;
-        if (lane == 0) pending = atomicAdd(&a.hdr->work_counter, 1u);
-        while (ok) {
-            const unsigned item = __shfl_sync(0xFFFFFFFFu, pending, 0);
-            if (item >= n_items) break;
-            if (lane == 0) pending = atomicAdd(&a.hdr->work_counter, 1u);   // in flight while this item is processed
+        if (lane == 0 && item < n_items) pending = n_warps + atomicAdd(&a.hdr->work_counter, 1u);
+        while (ok && item < n_items) {
             const int cblk = (int)(item / n_base);
             const unsigned base = item - (unsigned)cblk * n_base;
             ok = base < n_chunks ? do_chunk((int)base, cblk) : do_rows((int)(base - n_chunks), cblk);
+            item = __shfl_sync(0xFFFFFFFFu, pending, 0);
+            if (lane == 0 && item < n_items) pending = n_warps + atomicAdd(&a.hdr->work_counter, 1u);   // in flight during the next item
         }
         if (!ok) {
             // a wait gave up: let every copy this warp has issued land before the CTA's shared memory goes away
