@@ -448,15 +448,25 @@ struct WarpPipe {
         // grid starts up); later ones come from the counter, fetched one item ahead.
         const unsigned n_warps = gridDim.x * (unsigned)kPipeWarps;
         unsigned item = blockIdx.x * (unsigned)kPipeWarps + (unsigned)warp_id();
-        bool ok = true;
-        unsigned pending = 0;
-        if (lane == 0 && item < n_items) pending = n_warps + atomicAdd(&a.hdr->work_counter, 1u);
+        // While plenty of items are left, the next item is claimed one item ahead, so its number is
+        // back from the counter before it is needed.  Near the end that would leave some warps with
+        // an extra item in hand while others have run dry: then a warp claims only when it is out of work.
+        bool ok = true, lazy = n_items < 2u * n_warps;
+        unsigned pending = 0xFFFFFFFFu;
+        if (lane == 0 && item < n_items && !lazy) pending = n_warps + atomicAdd(&a.hdr->work_counter, 1u);
         while (ok && item < n_items) {
             const int cblk = (int)(item / n_base);
             const unsigned base = item - (unsigned)cblk * n_base;
             ok = base < n_chunks ? do_chunk((int)base, cblk) : do_rows((int)(base - n_chunks), cblk);
-            item = __shfl_sync(0xFFFFFFFFu, pending, 0);
-            if (lane == 0 && item < n_items) pending = n_warps + atomicAdd(&a.hdr->work_counter, 1u);   // in flight during the next item
+            if (lazy) {
+                unsigned it = 0;
+                if (lane == 0) it = n_warps + atomicAdd(&a.hdr->work_counter, 1u);
+                item = __shfl_sync(0xFFFFFFFFu, it, 0);
+            } else {
+                item = __shfl_sync(0xFFFFFFFFu, pending, 0);
+                if (item < n_items && n_items - item < 2u * n_warps) lazy = true;
+                if (lane == 0 && item < n_items && !lazy) pending = n_warps + atomicAdd(&a.hdr->work_counter, 1u);
+            }
         }
         if (!ok) {
             // a wait gave up: let every copy this warp has issued land before the CTA's shared memory goes away
