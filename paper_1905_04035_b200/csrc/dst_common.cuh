@@ -125,6 +125,7 @@ struct MainArgs {
     int ncb;         // column blocks per row
     int slot_bytes;
     int n_slots;
+    int precopied;   // rows below this number already hold dense_in (or zeros): those nobody names are left alone
 };
 
 // How the row-reduction kernel cuts rows into column blocks and shared memory into slots.
@@ -223,6 +224,10 @@ struct FrontParams {
     unsigned* node_cnt;
     long long vocab;
     int n_total, vocab_pad, chunk, batch_units, batch_max, nodecnt_words;
+    const void* copy_src;      // with copy_clusters > 0: dense_in, or nullptr to fill out with zeros
+    void* copy_dst;            // out
+    long long copy_bytes;      // vocab * d * sizeof(out element), a multiple of 16
+    int copy_clusters;         // extra clusters that fill out while the first one does the index work
 };
 cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStream_t stream);
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,

@@ -41,6 +41,9 @@ struct FrontArgs {
     int n_total, vocab_pad, chunk, batch_units, batch_max, nodecnt_words;
     int lw;                    // entries per warp (multiple of 32); a CTA's slice of the sorted order holds 32 * lw
     int rpt;                   // vocabulary rows per thread in the scan; a CTA's slice of count[] holds 1024 * rpt
+    const uint4* copy_src;     // clusters after the first: out = dense_in (or zeros), 16 bytes per thread and step
+    uint4* copy_dst;
+    long long copy_vecs;
 };
 
 constexpr int kFrontWarps = kFrontThreads / 32;
@@ -113,6 +116,27 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
     __shared__ int s_before[6], s_grand[6];
     __shared__ int s_maxseg[kFrontWarps];
 
+    if (blockIdx.x >= (unsigned)kClusterCtas) {
+        // Not the index cluster: meanwhile give every output row its dense_in row (or zeros).  The rows
+        // that do get contributions are rewritten by the row-reduction kernel; for a batch of a few
+        // thousand tokens against a vocabulary of tens of thousands that is a small part of the rows,
+        // and this copy, most of the bytes of the whole operation, hides the index work entirely.
+        const long long stride = (long long)(gridDim.x - kClusterCtas) * kFrontThreads;
+        long long i = (long long)(blockIdx.x - kClusterCtas) * kFrontThreads + threadIdx.x;
+        if (f.copy_src) {
+            for (; i + 7 * stride < f.copy_vecs; i += 8 * stride) {
+                uint4 v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = __ldcs(f.copy_src + i + q * stride);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) __stcs(f.copy_dst + i + q * stride, v[q]);
+            }
+            for (; i < f.copy_vecs; i += stride) __stcs(f.copy_dst + i, __ldcs(f.copy_src + i));
+        } else {
+            for (; i < f.copy_vecs; i += stride) __stcs(f.copy_dst + i, make_uint4(0u, 0u, 0u, 0u));
+        }
+        return;
+    }
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const int lane = lane_id(), warp = warp_id();
@@ -358,6 +382,9 @@ cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStrea
     f.unique_rows = p.unique_rows; f.counts_out = p.counts_out; f.result = p.result; f.batches = p.batches;
     f.node_cnt = p.node_cnt; f.vocab = p.vocab; f.n_total = p.n_total; f.vocab_pad = p.vocab_pad; f.chunk = p.chunk;
     f.batch_units = p.batch_units; f.batch_max = p.batch_max; f.nodecnt_words = p.nodecnt_words;
+    f.copy_src = static_cast<const uint4*>(p.copy_src); f.copy_dst = static_cast<uint4*>(p.copy_dst);
+    f.copy_vecs = p.copy_bytes / 16;
+    const int grid = kClusterCtas * (1 + (p.copy_clusters > 0 ? p.copy_clusters : 0));
     const int per_warp = (p.n_total + kClusterCtas * kFrontWarps - 1) / (kClusterCtas * kFrontWarps);
     f.lw = (per_warp + 31) / 32 * 32;
     if (f.lw < 32) f.lw = 32;
@@ -370,11 +397,11 @@ cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStrea
     if (index_type == DST_I64) {
         e = cudaFuncSetAttribute(k_front_cluster<long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k_front_cluster<long long><<<kClusterCtas, kFrontThreads, smem, stream>>>(f);
+        k_front_cluster<long long><<<grid, kFrontThreads, smem, stream>>>(f);
     } else {
         e = cudaFuncSetAttribute(k_front_cluster<int>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k_front_cluster<int><<<kClusterCtas, kFrontThreads, smem, stream>>>(f);
+        k_front_cluster<int><<<grid, kFrontThreads, smem, stream>>>(f);
     }
     return cudaGetLastError();
 }

@@ -429,7 +429,9 @@ struct WarpPipe {
                 } else {
                     b.y = v0 + i;
                     b.kind = kUnitFinal | (ci == 0 ? kUnitCopy : 0);
-                    if (a.dense_in) {
+                    if (ci == 0 && b.y < a.precopied) {
+                        b.kind = 0;                       // the row already holds its dense_in row (or zeros)
+                    } else if (a.dense_in) {
                         b.src = static_cast<const OT*>(a.dense_in) + (long long)b.y * a.d + cb;
                         b.bytes = (unsigned)(wcols * (long long)sizeof(OT));
                     }
@@ -554,8 +556,18 @@ static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaSt
     }
     const PipeShape ps = pipe_shape((int)sizeof(VT), (int)sizeof(OT), a.d);
     a.W = ps.W; a.ncb = ps.ncb; a.slot_bytes = ps.slot_bytes; a.n_slots = ps.n_slots;
-    const size_t smem = size_t(kPipeHeaderReserve) + size_t(kPipeWarps) * size_t(ps.n_slots) * size_t(ps.slot_bytes);
-    const int grid = sm_count * ps.ctas_per_sm;
+    int ctas_per_sm = ps.ctas_per_sm;
+    if (false && a.precopied && a.n_slots > 3) {
+        // Pre-filled output: few bytes left to move, bound by the latency of a work item: shallower rings,
+        // more warps.
+        a.n_slots = 3;
+        const int per_cta = kPipeHeaderReserve + kPipeWarps * a.n_slots * ps.slot_bytes + 1024 + 256;
+        ctas_per_sm = kSmemPerSm / per_cta;
+        if (ctas_per_sm > 3) ctas_per_sm = 3;      // what the kernel's registers allow
+        if (ctas_per_sm < ps.ctas_per_sm) ctas_per_sm = ps.ctas_per_sm;
+    }
+    const size_t smem = size_t(kPipeHeaderReserve) + size_t(kPipeWarps) * size_t(a.n_slots) * size_t(ps.slot_bytes);
+    const int grid = sm_count * ctas_per_sm;
     constexpr int kMaxK = sizeof(VT) == 4 ? 8 : 4;
     if (ps.K == 1) return launch_pipe<VT, OT, 1>(a, grid, smem, stream);
     if (ps.K == 2) return launch_pipe<VT, OT, 2>(a, grid, smem, stream);

@@ -58,12 +58,16 @@ def test_static_workspace_entry_point_matches_dst_densify_twice_in_a_row():
 
 
 def test_static_workspace_entry_point_refuses_shapes_beyond_its_array():
-    w = make_workload("big", scale=0.5)
-    assert dst.dst_workspace_bytes(w.n_rows_total, 1, w.d, w.vocab) > binding.STATIC_WORKSPACE_BYTES
-    idx, val = to_device(np.concatenate(w.indices), "i64"), to_device(np.concatenate(w.values), "f32")
-    out = torch.zeros(w.vocab, w.d, device="cuda")
+    # grow the input until a caller-owned workspace would have to be larger than the library's array
+    vocab, d, n = 5000, 256, 4096
+    while dst.dst_workspace_bytes(n, 1, d, vocab) <= binding.STATIC_WORKSPACE_BYTES:
+        n *= 2
+    rng = np.random.default_rng(0)
+    idx = torch.from_numpy(rng.integers(0, vocab, size=n)).cuda()
+    val = torch.from_numpy(rng.standard_normal((n, d)).astype(np.float32)).cuda()
+    out = torch.zeros(vocab, d, device="cuda")
     with pytest.raises(dst.DstError) as e:
-        dst.dst_densify_static(idx, val, w.d, w.vocab, None, out)
+        dst.dst_densify_static(idx, val, d, vocab, None, out)
     assert e.value.status == 3
     torch.cuda.synchronize()
     assert not out.any()        # nothing was enqueued
