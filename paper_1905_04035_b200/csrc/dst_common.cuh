@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "dst.h"
 
 namespace dst {
@@ -236,8 +238,28 @@ cudaError_t launch_scan(int index_type, const ScanParams& p, cudaStream_t stream
 cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,
                                cudaStream_t stream);
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor
+// in the stream is still running (once all of the predecessor's CTAs have called pdl_trigger), so the
+// launch latency and the kernel's prologue overlap with the predecessor's tail.  Every kernel calls
+// pdl_wait before it touches memory that an earlier kernel may still be writing.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 // ---- device helpers ---------------------------------------------------------
 #ifdef __CUDACC__
+// the kernels after this one in the stream may be scheduled now / wait for the kernels before this one
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
 __device__ __forceinline__ int warp_id() { return threadIdx.x >> 5; }
 

@@ -115,6 +115,8 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
     __shared__ int cta_sum[6];
     __shared__ int s_before[6], s_grand[6];
     __shared__ int s_maxseg[kFrontWarps];
+    pdl_trigger();
+    pdl_wait();
 
     if (blockIdx.x >= (unsigned)kClusterCtas) {
         // Not the index cluster: meanwhile give every output row its dense_in row (or zeros).  The rows
@@ -397,11 +399,11 @@ cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStrea
     if (index_type == DST_I64) {
         e = cudaFuncSetAttribute(k_front_cluster<long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k_front_cluster<long long><<<grid, kFrontThreads, smem, stream>>>(f);
+        return launch_pdl(k_front_cluster<long long>, dim3(grid), dim3(kFrontThreads), smem, stream, f);
     } else {
         e = cudaFuncSetAttribute(k_front_cluster<int>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k_front_cluster<int><<<grid, kFrontThreads, smem, stream>>>(f);
+        return launch_pdl(k_front_cluster<int>, dim3(grid), dim3(kFrontThreads), smem, stream, f);
     }
     return cudaGetLastError();
 }

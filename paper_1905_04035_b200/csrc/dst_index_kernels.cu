@@ -24,6 +24,8 @@ __global__ void __launch_bounds__(kSortThreads)
 k_prep(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, unsigned* __restrict__ digit_hist,
        unsigned* __restrict__ keys, SliceEntry* __restrict__ tab, long long vocab, int passes) {
     __shared__ unsigned dh[kMaxPasses * 256];
+    pdl_trigger();
+    pdl_wait();
 
     const SliceEntry& se = P.s[blockIdx.y];
     if (blockIdx.x == 0 && threadIdx.x == 0) tab[P.first + blockIdx.y] = se;
@@ -110,6 +112,8 @@ k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, c
     __shared__ unsigned bin_base[256];
     __shared__ unsigned wsum[kWarps];
     __shared__ unsigned s_tile;
+    pdl_trigger();
+    pdl_wait();
     if (threadIdx.x == 0) s_tile = atomicAdd(&hdr->ticket[pass], 1u);   // tiles start in id order
     for (int s = threadIdx.x; s < kWarps * 256; s += kSortThreads) (&wh[0][0])[s] = 0;
     __syncthreads();
@@ -186,6 +190,8 @@ k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, c
 __global__ void __launch_bounds__(256)
 k_bounds(const WsHeader* __restrict__ hdr, const unsigned* __restrict__ keys, unsigned* __restrict__ count,
          int capacity, int vocab) {
+    pdl_trigger();
+    pdl_wait();
     const int n = capacity - (int)hdr->n_bad;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
@@ -260,6 +266,8 @@ k_scan(const ScanArgs s) {
     __shared__ int s_tile;
     __shared__ int s_fail;
     WsHeader* hdr = s.hdr;
+    pdl_trigger();
+    pdl_wait();
     const int chunk = s.chunk, B = s.batch_units, vocab = s.vocab;
     IT* unique_rows = static_cast<IT*>(s.unique_rows);
     if (threadIdx.x == 0) {
@@ -423,33 +431,29 @@ cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeade
                         unsigned* keys, SliceEntry* tab, long long vocab, int passes, cudaStream_t stream) {
     dim3 grid(grid_x, P.n);
     if (index_type == DST_I64)
-        k_prep<long long><<<grid, kSortThreads, 0, stream>>>(P, hdr, digit_hist, keys, tab, vocab, passes);
+        return launch_pdl(k_prep<long long>, grid, dim3(kSortThreads), 0, stream, P, hdr, digit_hist, keys, tab, vocab, passes);
     else
-        k_prep<int><<<grid, kSortThreads, 0, stream>>>(P, hdr, digit_hist, keys, tab, vocab, passes);
-    return cudaGetLastError();
+        return launch_pdl(k_prep<int>, grid, dim3(kSortThreads), 0, stream, P, hdr, digit_hist, keys, tab, vocab, passes);
 }
 
 cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
                               unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
                               int pass, int capacity, cudaStream_t stream) {
-    k_radix_pass<<<n_tiles, kSortThreads, 0, stream>>>(hdr, in_keys, in_pos, out_keys, out_pos, digit_hist, desc,
-                                                       pass, capacity);
-    return cudaGetLastError();
+    return launch_pdl(k_radix_pass, dim3(n_tiles), dim3(kSortThreads), 0, stream, hdr, in_keys, in_pos, out_keys, out_pos,
+                      digit_hist, desc, pass, capacity);
 }
 
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
                           cudaStream_t stream) {
-    k_bounds<<<(capacity + 255) / 256, 256, 0, stream>>>(hdr, keys, count, capacity, vocab);
-    return cudaGetLastError();
+    return launch_pdl(k_bounds, dim3((capacity + 255) / 256), dim3(256), 0, stream, hdr, keys, count, capacity, vocab);
 }
 
 cudaError_t launch_scan(int index_type, const ScanParams& p, cudaStream_t stream) {
     const int n_tiles = (p.vocab_pad + kScanTile - 1) / kScanTile;
     ScanArgs s{p.hdr, p.count, p.offsets, p.heavy, p.unique_rows, p.counts_out, p.result, p.batches,
                p.scan_desc, p.vocab, p.vocab_pad, p.chunk, p.batch_units, n_tiles};
-    if (index_type == DST_I64) k_scan<long long><<<n_tiles, kScanThreads, 0, stream>>>(s);
-    else k_scan<int><<<n_tiles, kScanThreads, 0, stream>>>(s);
-    return cudaGetLastError();
+    if (index_type == DST_I64) return launch_pdl(k_scan<long long>, dim3(n_tiles), dim3(kScanThreads), 0, stream, s);
+    return launch_pdl(k_scan<int>, dim3(n_tiles), dim3(kScanThreads), 0, stream, s);
 }
 
 }  // namespace dst

@@ -495,7 +495,9 @@ k_reduce_rows(const __grid_constant__ MainArgs a) {
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    pdl_trigger();
     __syncthreads();
+    pdl_wait();       // everything above overlaps with the tail of the kernel before
     {
         char* my_ring = slot_base + (size_t)warp * (size_t)a.n_slots * (size_t)a.slot_bytes;
         WarpPipe<VT, OT, K> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort);
@@ -540,8 +542,7 @@ template <typename VT, typename OT, int K>
 static cudaError_t launch_pipe(const MainArgs& a, int grid, size_t smem, cudaStream_t stream) {
     cudaError_t e = cudaFuncSetAttribute(k_reduce_rows<VT, OT, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k_reduce_rows<VT, OT, K><<<grid, kPipeThreads, smem, stream>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(k_reduce_rows<VT, OT, K>, dim3(grid), dim3(kPipeThreads), smem, stream, a);
 }
 
 template <typename VT, typename OT>
