@@ -157,6 +157,15 @@ enum : int {
     kUnitChunkEnd = 8    // last entry of chunk y: store the partial row, climb the tree
 };
 
+constexpr int kTabCache = 64;       // slices whose table is copied into shared memory
+constexpr int kHeavyCache = 1024;   // heavy rows whose first chunk id is copied into shared memory
+struct CtaTables {
+    long long start[kTabCache];
+    unsigned long long values[kTabCache];
+    int chunk_base[kHeavyCache];
+    int n_heavy;
+};
+
 // A block of at most 32 units, one per lane.
 struct UnitBlock {
     const void* src;     // first byte to copy (nullptr: nothing to copy)
@@ -174,13 +183,16 @@ struct WarpPipe {
     const unsigned bars;      // shared address of this warp's first mbarrier (one per slot)
     char* const ring_ptr;     // generic address of the first slot
     volatile int* const abort_flag;
+    const CtaTables& tabs;    // this CTA's shared copies of the slice table and of the heavy rows' first chunk ids
+    HeavyInfo cur_heavy;      // the heavy row of the chunk item being processed
     int islot;                // slot the next issued unit goes to
     int cslot;                // slot of the next unit to consume
     unsigned cphase;          // bit s: parity to wait for on slot s
     unsigned issued_mask;     // slots with a copy that may still be in flight
 
-    __device__ WarpPipe(const MainArgs& args, unsigned ring_addr, unsigned bar_addr, char* ring_generic, volatile int* ab)
-        : a(args), lane(lane_id()), ring(ring_addr), bars(bar_addr), ring_ptr(ring_generic), abort_flag(ab), islot(0),
+    __device__ WarpPipe(const MainArgs& args, unsigned ring_addr, unsigned bar_addr, char* ring_generic, volatile int* ab,
+                        const CtaTables& t)
+        : a(args), lane(lane_id()), ring(ring_addr), bars(bar_addr), ring_ptr(ring_generic), abort_flag(ab), tabs(t), islot(0),
           cslot(0), cphase(0u), issued_mask(0u) {}
 
     __device__ __forceinline__ int col(int k) const { return (k * 32 + lane) * VC; }
@@ -200,6 +212,17 @@ struct WarpPipe {
         }
         issued_mask |= 1u << islot;
         islot = islot + 1 == a.n_slots ? 0 : islot + 1;
+    }
+
+    // position in the virtual concatenation -> address of that value row (slice table in shared memory)
+    __device__ __forceinline__ const VT* row_address(unsigned p) const {
+        if (a.R > kTabCache) return resolve_row<VT>(a, p);
+        int lo = 0, hi = a.R - 1;                  // largest r with start[r] <= p
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (tabs.start[mid] <= (long long)p) lo = mid; else hi = mid - 1;
+        }
+        return reinterpret_cast<const VT*>(tabs.values[lo]) + ((long long)p - tabs.start[lo]) * a.d;
     }
 
     __device__ __forceinline__ float* partial_row(int slot) const { return a.partials + (long long)slot * a.d; }
@@ -226,11 +249,18 @@ struct WarpPipe {
         }
     }
 
-    // Heavy row that owns chunk cid: the last h with heavy[h].chunk_base <= cid.  All lanes probe
-    // at once, so the table (a few hundred entries) is searched in two or three steps.
+    // Heavy row that owns chunk cid: the last h with heavy[h].chunk_base <= cid.
     __device__ __forceinline__ int find_heavy(int cid) const {
-        int lo = 0, hi = a.hdr->n_heavy;
-        while (hi - lo > 1) {
+        int lo = 0, hi = tabs.n_heavy;
+        if (hi <= kHeavyCache) {                     // the first chunk ids are in shared memory
+            --hi;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (tabs.chunk_base[mid] <= cid) lo = mid; else hi = mid - 1;
+            }
+            return lo;
+        }
+        while (hi - lo > 1) {                        // all lanes probe at once
             const int step = (hi - lo + 31) / 32;
             const int idx = lo + lane * step;
             const bool le = idx < hi && __ldg(&a.heavy[idx].chunk_base) <= cid;
@@ -240,9 +270,10 @@ struct WarpPipe {
         }
         return lo;
     }
-    __device__ __forceinline__ ChunkDesc chunk_of(int cid) const {
+    __device__ __forceinline__ ChunkDesc chunk_of(int cid) {
         const int h = find_heavy(cid);
         const HeavyInfo hi = a.heavy[h];
+        cur_heavy = hi;
         const int k = cid - hi.chunk_base;
         return ChunkDesc{hi.row, hi.begin + k * a.chunk, min(a.chunk, hi.count - k * a.chunk), h};
     }
@@ -250,7 +281,7 @@ struct WarpPipe {
     // The chunk's sum is in acc: store it as a partial row and climb the combine tree while this
     // warp is the last child to arrive.
     __device__ void finish_chunk(Acc<VC> (&acc)[K], int cid, int cblk) const {
-        const HeavyInfo hi = a.heavy[find_heavy(cid)];
+        const HeavyInfo hi = cur_heavy;
         const long long cb = (long long)cblk * a.W;
         const int wcols = (int)min((long long)a.W, a.d - cb);
         {
@@ -376,7 +407,7 @@ struct WarpPipe {
             UnitBlock b{nullptr, 0u, 0, cid};
             if (q < cd.len) {
                 const unsigned p = a.perm[cd.begin + q];
-                if (p < (unsigned)a.n_total) { b.src = resolve_row<VT>(a, p) + cb; b.bytes = bytes; b.kind = kUnitAdd; }
+                if (p < (unsigned)a.n_total) { b.src = row_address(p) + cb; b.bytes = bytes; b.kind = kUnitAdd; }
                 if (q == cd.len - 1) b.kind |= kUnitChunkEnd;
             }
             if (!run_block(acc, b, min(32, cd.len - base), cblk)) return false;
@@ -422,7 +453,7 @@ struct WarpPipe {
                 if (e < ci) {
                     const unsigned p = a.perm[oi + e];
                     if (p < (unsigned)a.n_total) {
-                        b.src = resolve_row<VT>(a, p) + cb;
+                        b.src = row_address(p) + cb;
                         b.bytes = (unsigned)(wcols * (long long)sizeof(VT));
                         b.kind = kUnitAdd;
                     }
@@ -487,6 +518,7 @@ __global__ void __launch_bounds__(kPipeThreads)
 k_reduce_rows(const __grid_constant__ MainArgs a) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ int s_abort;
+    __shared__ CtaTables tabs;
     unsigned long long* bar_base = reinterpret_cast<unsigned long long*>(smem_raw);
     char* slot_base = reinterpret_cast<char*>(smem_raw) + kPipeHeaderReserve;
     const int warp = warp_id();
@@ -496,11 +528,23 @@ k_reduce_rows(const __grid_constant__ MainArgs a) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     pdl_trigger();
-    __syncthreads();
     pdl_wait();       // everything above overlaps with the tail of the kernel before
+    if (a.R <= kTabCache) {
+        for (int r = threadIdx.x; r < a.R; r += kPipeThreads) {
+            tabs.start[r] = a.tab[r].start;
+            tabs.values[r] = reinterpret_cast<unsigned long long>(a.tab[r].values);
+        }
+    }
+    {
+        const int nh = a.hdr->n_heavy;
+        if (threadIdx.x == 0) tabs.n_heavy = nh;
+        if (nh <= kHeavyCache)
+            for (int h = threadIdx.x; h < nh; h += kPipeThreads) tabs.chunk_base[h] = a.heavy[h].chunk_base;
+    }
+    __syncthreads();
     {
         char* my_ring = slot_base + (size_t)warp * (size_t)a.n_slots * (size_t)a.slot_bytes;
-        WarpPipe<VT, OT, K> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort);
+        WarpPipe<VT, OT, K> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort, tabs);
         // after a failed wait in an earlier kernel the tables are not to be trusted: touch nothing
         if (*reinterpret_cast<volatile int*>(&a.hdr->status) != DST_ERR_TIMEOUT) pipe.run();
     }
