@@ -11,8 +11,8 @@ namespace dst {
 static thread_local cudaEvent_t t_ev_before = nullptr, t_ev_after = nullptr;
 static std::atomic<long long> g_launches{0};
 
-// bytes the copy clusters of the small-input path move while its index cluster works (about 30 us)
-constexpr double kPrecopyBytes = 160e6;
+// bytes the copy clusters of the small-input path move while its index cluster works (about 35 us)
+constexpr double kPrecopyBytes = 200e6;
 
 static size_t index_size(int t) { return t == DST_I64 ? 8 : 4; }
 static size_t dtype_size(int t) { return t == DST_F32 ? 4 : 2; }
