@@ -184,6 +184,54 @@ def test_dtype_pairs(vt, ot):
     assert_parity(w, run_library(w))
 
 
+# ---------------------------------------------------------------------------
+# the two index paths and the pre-filled output of the small-input path
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("n,vocab,R", [
+    (65535, 65536, 1),      # largest input of the one-kernel index path
+    (65536, 65536, 1),      # one more row: general path
+    (3000, 65537, 1),       # one more vocabulary row: general path
+    (3000, 65536, 64),      # most slices the one-kernel path takes
+    (3000, 65536, 65),      # one more slice: general path
+    (3000, 1000, 3),        # small path, more rows than vocabulary: nothing is pre-filled
+])
+def test_index_path_boundaries(n, vocab, R):
+    ns = [n // R + (1 if r < n % R else 0) for r in range(R)]
+    hot = lambda rng, k: np.where(rng.random(k) < 0.3, vocab - 1, rng.integers(0, vocab, size=k))
+    w = _custom(vocab, 64, ns, idx_fn=hot)
+    a = run_library(w, mode="concat")
+    assert_parity(w, a)
+    assert np.array_equal(raw_bits(a.out), raw_bits(run_library(w, mode="single").out))
+
+
+@pytest.mark.parametrize("d,with_dense,in_place", [(64, True, False), (2056, True, False), (512, False, False),
+                                                   (512, True, True), (4096, True, True)])
+def test_prefilled_output_small_inputs(d, with_dense, in_place):
+    # few rows against the vocabulary: most of out is written by the index kernel's extra clusters
+    vocab = 40000 if d <= 512 else 6000
+    hot = lambda rng, k: np.where(rng.random(k) < 0.4, 7, rng.integers(0, vocab, size=k))
+    w = _custom(vocab, d, [1500, 0, 700], idx_fn=hot, with_dense=with_dense, std=0.5)
+    run = run_library(w, in_place=in_place)
+    if in_place:
+        orc = oracle_of(w)
+        assert np.all(np.abs(to_numpy_f64(run.out) - orc.acc) <= 1e-5 * orc.mag + 1e-7)
+        assert np.array_equal(raw_bits(run.out), raw_bits(run_library(w).out))
+    else:
+        assert_parity(w, run)
+
+
+def test_prefilled_output_bf16_and_out_of_range():
+    vocab = 50000
+    def idx(rng, k):
+        ix = rng.integers(0, vocab, size=k)
+        ix[::9] = vocab + rng.integers(0, 100, size=ix[::9].shape[0])
+        return ix
+    w = _custom(vocab, 256, [4000], idx_fn=idx, value_dtype="bf16", out_dtype="bf16", index_dtype="i32")
+    assert_parity(w, run_library(w))
+    w = _custom(vocab, 256, [4000], idx_fn=idx, value_dtype="bf16", out_dtype="f32", with_dense=False)
+    assert_parity(w, run_library(w))
+
+
 def test_many_slices_use_several_histogram_launches():
     ns = [int(x) for x in np.random.default_rng(1).integers(0, 200, size=150)]
     w = _custom(1500, 128, ns)
