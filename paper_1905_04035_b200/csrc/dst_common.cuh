@@ -143,7 +143,7 @@ inline PipeShape pipe_shape(int value_size, int out_size, int64_t d) {
     const int widest = value_size > out_size ? value_size : out_size;
     p.slot_bytes = (p.W * widest + 127) / 128 * 128;
     p.n_slots = kPipeSlots;
-    const int per_cta = kPipeHeaderReserve + kPipeWarps * p.n_slots * p.slot_bytes + 1024;   // + the driver's reserve
+    const int per_cta = kPipeHeaderReserve + kPipeWarps * p.n_slots * p.slot_bytes + 1024 + 5376;   // + the driver's reserve + the kernel's static tables
     int c = kSmemPerSm / per_cta;
     p.ctas_per_sm = c < 1 ? 1 : (c > 8 ? 8 : c);
     return p;

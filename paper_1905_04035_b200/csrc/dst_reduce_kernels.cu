@@ -227,25 +227,29 @@ struct WarpPipe {
 
     __device__ __forceinline__ float* partial_row(int slot) const { return a.partials + (long long)slot * a.d; }
 
-    // acc = child[0] + child[1] + ... in index order
+    // acc = child[0] + child[1] + ... in index order (half of the column groups at a time, to save registers)
     __device__ __forceinline__ void sum_children(Acc<VC> (&acc)[K], int first_slot, int n, long long cb, int wcols) const {
+        constexpr int KH = K >= 4 ? K / 2 : K;
 #pragma unroll
-        for (int k = 0; k < K; ++k) zero(acc[k]);
-        for (int c = 0; c < n; c += 2) {
-            const float* pa = partial_row(first_slot + c) + cb;
-            const float* pb = (c + 1 < n) ? partial_row(first_slot + c + 1) + cb : nullptr;
-            Acc<VC> va[K], vb[K];
+        for (int h0 = 0; h0 < K; h0 += KH) {
 #pragma unroll
-            for (int k = 0; k < K; ++k) {
-                const int cc = col(k);
-                zero(va[k]); zero(vb[k]);
-                if (cc < wcols) {
-                    load_partial(pa + cc, va[k]);
-                    if (pb) load_partial(pb + cc, vb[k]);
+            for (int k = 0; k < KH; ++k) zero(acc[h0 + k]);
+            for (int c = 0; c < n; c += 2) {
+                const float* pa = partial_row(first_slot + c) + cb;
+                const float* pb = (c + 1 < n) ? partial_row(first_slot + c + 1) + cb : nullptr;
+                Acc<VC> va[KH], vb[KH];
+#pragma unroll
+                for (int k = 0; k < KH; ++k) {
+                    const int cc = col(h0 + k);
+                    zero(va[k]); zero(vb[k]);
+                    if (cc < wcols) {
+                        load_partial(pa + cc, va[k]);
+                        if (pb) load_partial(pb + cc, vb[k]);
+                    }
                 }
-            }
 #pragma unroll
-            for (int k = 0; k < K; ++k) { add(acc[k], va[k]); add(acc[k], vb[k]); }
+                for (int k = 0; k < KH; ++k) { add(acc[h0 + k], va[k]); add(acc[h0 + k], vb[k]); }
+            }
         }
     }
 
@@ -514,7 +518,7 @@ struct WarpPipe {
 };
 
 template <typename VT, typename OT, int K>
-__global__ void __launch_bounds__(kPipeThreads)
+__global__ void __launch_bounds__(kPipeThreads, sizeof(VT) == 2 ? 4 : 2)
 k_reduce_rows(const __grid_constant__ MainArgs a) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ int s_abort;
