@@ -35,6 +35,10 @@ from paper_1905_04035_b200.workloads import make_workload  # noqa: E402
 L2_BYTES = 126 * 1024 * 1024
 SIZEOF = {"f32": 4, "bf16": 2, "i32": 4, "i64": 8}
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the row-reduction kernel, from an ncu capture of
+# this command on the full-size workload (1 pass; profiles/k_reduce_rows_r64_full_dram_bytes.md).  Only for the
+# workloads that were captured with the kernel as it stands.
+KERNEL_DRAM_TRAFFIC = {"r64": 2.85e9 + 138.6e6}
 ALL_CONFIGS = ("tiny", "base", "big", "r64", "sweep_uniform", "sweep_zipf", "sweep_same")
 
 
@@ -471,7 +475,8 @@ def main():
             "eager_ms_per_step": head["eager_ms_per_step"],
             "rows_per_s": agg["rows_per_s"], "frac_of_hbm_peak": agg["gbs"] / world / head["peak_gbs"],
             "roofline": {"bound": "hbm", "achieved": head["reduce_kernel_gbs"], "peak": head["peak_gbs"],
-                         "unit": "GB/s", "frac": head["reduce_kernel_frac"], "traffic": None,
+                         "unit": "GB/s", "frac": head["reduce_kernel_frac"],
+                         "traffic": KERNEL_DRAM_TRAFFIC.get(args.workload) if args.scale == 1.0 else None,
                          "kernel": "k_reduce_rows", "of": head["peak_source"],
                          "kernel_ms": head["reduce_kernel_ms"]},
             "e2e": e2e, "gpu_launches": head["launches"], "clocks": head["clocks"],

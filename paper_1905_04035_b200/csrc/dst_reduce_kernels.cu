@@ -227,9 +227,9 @@ struct WarpPipe {
 
     __device__ __forceinline__ float* partial_row(int slot) const { return a.partials + (long long)slot * a.d; }
 
-    // acc = child[0] + child[1] + ... in index order (half of the column groups at a time, to save registers)
+    // acc = child[0] + child[1] + ... in index order (bf16: half of the column groups at a time, to save registers)
     __device__ __forceinline__ void sum_children(Acc<VC> (&acc)[K], int first_slot, int n, long long cb, int wcols) const {
-        constexpr int KH = K >= 4 ? K / 2 : K;
+        constexpr int KH = (sizeof(VT) == 2 && K >= 4) ? K / 2 : K;   // the bf16 variants run at 128 registers
 #pragma unroll
         for (int h0 = 0; h0 < K; h0 += KH) {
 #pragma unroll
