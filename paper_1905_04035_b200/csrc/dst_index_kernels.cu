@@ -49,12 +49,8 @@ k_prep(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, unsigne
         const unsigned key = ok ? (unsigned)v : kInvalidKey;
         if (in) keys[se.start + i] = key;
         bad += in && !ok;
-        // equal digits inside the warp are added once (frequent rows would otherwise serialise)
-        for (int p = 0; p < passes; ++p) {
-            const unsigned dg = (key >> (8 * p)) & 255u;
-            const unsigned m = match_digit(dg, ok);
-            if (ok && lane == __ffs(m) - 1) atomicAdd(&dh[p * 256 + dg], (unsigned)__popc(m));
-        }
+        if (ok)
+            for (int p = 0; p < passes; ++p) atomicAdd(&dh[p * 256 + ((key >> (8 * p)) & 255u)], 1u);
     }
     __syncthreads();
     for (int s = threadIdx.x; s < passes * 256; s += kSortThreads) {
