@@ -11,9 +11,6 @@ namespace dst {
 static thread_local cudaEvent_t t_ev_before = nullptr, t_ev_after = nullptr;
 static std::atomic<long long> g_launches{0};
 
-// bytes the copy clusters of the small-input path move while its index cluster works (about 35 us)
-constexpr double kPrecopyBytes = 200e6;
-
 static size_t index_size(int t) { return t == DST_I64 ? 8 : 4; }
 static size_t dtype_size(int t) { return t == DST_F32 ? 4 : 2; }
 
@@ -79,7 +76,7 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         if (slices[r].n_rows > 0 && !aligned16(slices[r].values)) vector_ok = false;
 
     const unsigned* perm = pos[L.passes & 1];
-    int64_t precopied = 0;
+    bool compact = false;
     const bool small = n_total <= kFrontMaxRows && vocab <= 65536 && R <= kHistSlices;
     if (small) {
         // small input: one cluster kernel does the whole index side and clears its own tables
@@ -96,18 +93,17 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         fp.node_cnt = nodecnt; fp.vocab = vocab; fp.n_total = int(n_total); fp.vocab_pad = int(L.vocab_pad);
         fp.chunk = L.chunk; fp.batch_units = L.batch_units; fp.batch_max = int(L.batch_max);
         fp.nodecnt_words = int((L.off_batches - L.off_nodecnt) / 4);
-        // Few input rows against the vocabulary: most output rows are plain copies of dense_in.  Extra
-        // clusters of the same launch write the first `precopied` of them while the first cluster does the
-        // index work (about as many rows as fit into that time); the row-reduction kernel then leaves
-        // those rows alone unless they were named.  In place there is nothing to copy.
-        if (vector_ok && n_total <= vocab) {
-            const double row_bytes = double(d) * double(dtype_size(opts->out_type));
-            const double rows = out == dense_in ? double(vocab) : kPrecopyBytes / ((dense_in ? 2.0 : 1.0) * row_bytes);
-            precopied = rows >= double(vocab) ? int64_t(vocab) : int64_t(rows);
-        }
+        // No more input rows than vocabulary rows: most output rows are plain copies of dense_in.  Extra
+        // clusters of the same launch write out = dense_in (or zeros) for every row while the first cluster
+        // does the index work; the row-reduction kernel then visits only the rows that were named (and
+        // reads and writes those a second time).  In place there is nothing to copy.
+        compact = vector_ok && n_total <= vocab;
+        fp.compact = compact ? 1 : 0;
+        fp.urow = reinterpret_cast<int*>(ws + L.off_urow);
+        fp.uoff = reinterpret_cast<int*>(ws + L.off_uoff);
         fp.copy_src = dense_in; fp.copy_dst = out;
-        fp.copy_bytes = precopied * d * int64_t(dtype_size(opts->out_type));
-        fp.copy_clusters = precopied > 0 && out != dense_in ? (sm_count() - kClusterCtas) / kClusterCtas : 0;
+        fp.copy_bytes = int64_t(vocab) * d * int64_t(dtype_size(opts->out_type));
+        fp.copy_clusters = compact && out != dense_in ? (sm_count() - kClusterCtas) / kClusterCtas : 0;
         if (launch_front_cluster(opts->index_type, fp, stream) != cudaSuccess) return DST_ERR_CUDA;
         ++g_launches;
         perm = pos[0];
@@ -160,7 +156,9 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     a.result = result; a.d = d; a.vocab = int(vocab); a.n_total = int(n_total); a.R = R; a.chunk = L.chunk;
     a.chunk_max = int(L.chunk_max); a.upper_max = int(L.upper_max);
     a.W = a.ncb = a.slot_bytes = a.n_slots = 0;   // set by the launcher
-    a.precopied = int(precopied);
+    a.compact = compact ? 1 : 0;
+    a.urow = reinterpret_cast<const int*>(ws + L.off_urow);
+    a.uoff = reinterpret_cast<const int*>(ws + L.off_uoff);
     if (t_ev_before && cudaEventRecord(t_ev_before, stream) != cudaSuccess) return DST_ERR_CUDA;
     if (launch_reduce_rows(a, opts->value_type, opts->out_type, vector_ok, sm_count(), stream) != cudaSuccess)
         return DST_ERR_CUDA;

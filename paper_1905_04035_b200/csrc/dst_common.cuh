@@ -99,7 +99,7 @@ struct Layout {
     int R, chunk, passes, batch_units;
     int64_t n_tiles, vocab_pad, heavy_max, chunk_max, upper_max, batch_max;
     size_t off_header, off_count, off_digit, off_desc, off_nodecnt, off_batches, off_scandesc, zero_bytes;
-    size_t off_offsets, off_keys[2], off_pos[2], off_tab, off_heavy, off_partials;
+    size_t off_offsets, off_keys[2], off_pos[2], off_tab, off_heavy, off_partials, off_urow, off_uoff;
     size_t total;
 };
 
@@ -110,7 +110,9 @@ struct MainArgs {
     const unsigned* perm;
     const SliceEntry* tab;
     const HeavyInfo* heavy;
-    const int2* batches;   // per row batch: first row + 1 (0: empty batch), last row + 1
+    const int2* batches;   // per row batch: first row + 1 (0: empty batch), last row + 1; `compact`: numbers in urow[]
+    const int* urow;       // compact: the named rows, ascending
+    const int* uoff;       // compact: first entry of each named row in perm[], then the number of entries
     unsigned* node_cnt;
     float* partials;
     const void* dense_in;
@@ -127,7 +129,7 @@ struct MainArgs {
     int ncb;         // column blocks per row
     int slot_bytes;
     int n_slots;
-    int precopied;   // rows below this number already hold dense_in (or zeros): those nobody names are left alone
+    int compact;     // out already holds dense_in (or zeros) everywhere: the row batches list only the named rows
 };
 
 // How the row-reduction kernel cuts rows into column blocks and shared memory into slots.
@@ -192,6 +194,11 @@ inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab, i
     L.off_pos[1] = take(size_t(n_rows) * 4);
     L.off_tab = take(size_t(R > 0 ? R : 1) * sizeof(SliceEntry));
     L.off_heavy = take(size_t(L.heavy_max + 1) * sizeof(HeavyInfo));
+    {
+        const int64_t cap = (n_rows < vocab ? n_rows : vocab) + 2;
+        L.off_urow = take(size_t(cap) * 4);
+        L.off_uoff = take(size_t(cap) * 4);
+    }
     L.off_partials = take(size_t(L.chunk_max + L.upper_max) * size_t(d) * 4);
     L.total = o;
     return L;
@@ -229,6 +236,9 @@ struct FrontParams {
     unsigned* node_cnt;
     long long vocab;
     int n_total, vocab_pad, chunk, batch_units, batch_max, nodecnt_words;
+    int compact;               // list only the named rows in the row batches (and in urow / uoff)
+    int* urow;
+    int* uoff;
     const void* copy_src;      // with copy_clusters > 0: dense_in, or nullptr to fill out with zeros
     void* copy_dst;            // out
     long long copy_bytes;      // vocab * d * sizeof(out element), a multiple of 16

@@ -19,6 +19,8 @@
 // R <= kHistSlices (the slice table travels as a kernel parameter).
 #include <cooperative_groups.h>
 
+#include <atomic>
+
 #include "dst_common.cuh"
 
 namespace cg = cooperative_groups;
@@ -36,6 +38,9 @@ struct FrontArgs {
     int* counts_out;
     dst_result_t* result;
     int2* batches;
+    int* urow;
+    int* uoff;
+    int compact;
     unsigned* node_cnt;
     long long vocab;
     int n_total, vocab_pad, chunk, batch_units, batch_max, nodecnt_words;
@@ -153,7 +158,7 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
 
     // ---- clear what must start at zero
     for (int i = threadIdx.x; i < Vs; i += kFrontThreads) cnt[i] = 0;
-    for (int i = gt; i < f.batch_max; i += kAllThreads) f.batches[i] = make_int2(0, 0);
+    for (int i = gt; i < f.batch_max; i += kAllThreads) f.batches[i] = make_int2(f.compact ? 0x7FFFFFFF : 0, 0);
     for (int i = gt; i < f.nodecnt_words; i += kAllThreads) f.node_cnt[i] = 0;
     if (rank == 0) {
         if (threadIdx.x < (int)(sizeof(WsHeader) / 4)) reinterpret_cast<unsigned*>(hdr)[threadIdx.x] = 0;
@@ -257,7 +262,7 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
         const int cc = c[q];
         mine.v[0] += cc;
         mine.v[1] += cc > 0;
-        if (q < f.rpt && e0 + q < vocab) mine.v[5] += row_units(cc, chunk);
+        if (q < f.rpt && e0 + q < vocab && !(f.compact && cc == 0)) mine.v[5] += row_units(cc, chunk);
         if (cc > chunk) {
             const int n = (cc + chunk - 1) / chunk;
             mine.v[2] += 1; mine.v[3] += n; mine.v[4] += upper_nodes(n);
@@ -337,6 +342,17 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
                 if (cc > 0) {
                     if (unique_rows) unique_rows[run.v[1]] = (IT)v;
                     if (f.counts_out) f.counts_out[run.v[1]] = cc;
+                    if (f.compact) {
+                        // the row batches list named rows only: row number and first entry by rank among them
+                        const int u = run.v[1];
+                        f.urow[u] = v;
+                        f.uoff[u] = run.v[0];
+                        const int cost = row_units(cc, chunk);
+                        atomicMin(&f.batches[b].x, u + 1);
+                        atomicMax(&f.batches[b].y, u + 1);
+                        rem += cost;
+                        if (rem >= B) { b += rem / B; rem %= B; }
+                    }
                     run.v[1] += 1;
                 }
                 if (cc > chunk) {
@@ -346,7 +362,7 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
                     run.v[2] += 1; run.v[3] += n; run.v[4] += upper_nodes(n);
                 }
                 run.v[0] += cc;
-                if (v < vocab) {
+                if (v < vocab && !f.compact) {
                     // light work items: row v belongs to batch floor(units before v / batch size)
                     const int cost = row_units(cc, chunk);
                     if (v == 0 || prev_cost > rem) f.batches[b].x = v + 1;
@@ -361,6 +377,7 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
     cluster.sync();       // all tables and the header's max_segment are written; nobody reads a peer's shared memory after this
     if (rank == 0 && threadIdx.x == 0) {
         f.offsets[f.vocab_pad] = s_grand[0];
+        if (f.compact) f.uoff[s_grand[1]] = s_grand[0];
         hdr->n_valid = s_grand[0];
         hdr->n_unique = s_grand[1];
         hdr->n_heavy = s_grand[2];
@@ -382,11 +399,11 @@ cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStrea
     FrontArgs f;
     f.P = p.P; f.hdr = p.hdr; f.tab = p.tab; f.perm = p.perm; f.offsets = p.offsets; f.heavy = p.heavy;
     f.unique_rows = p.unique_rows; f.counts_out = p.counts_out; f.result = p.result; f.batches = p.batches;
+    f.urow = p.urow; f.uoff = p.uoff; f.compact = p.compact;
     f.node_cnt = p.node_cnt; f.vocab = p.vocab; f.n_total = p.n_total; f.vocab_pad = p.vocab_pad; f.chunk = p.chunk;
     f.batch_units = p.batch_units; f.batch_max = p.batch_max; f.nodecnt_words = p.nodecnt_words;
     f.copy_src = static_cast<const uint4*>(p.copy_src); f.copy_dst = static_cast<uint4*>(p.copy_dst);
     f.copy_vecs = p.copy_bytes / 16;
-    const int grid = kClusterCtas * (1 + (p.copy_clusters > 0 ? p.copy_clusters : 0));
     const int per_warp = (p.n_total + kClusterCtas * kFrontWarps - 1) / (kClusterCtas * kFrontWarps);
     f.lw = (per_warp + 31) / 32 * 32;
     if (f.lw < 32) f.lw = 32;
@@ -396,16 +413,43 @@ cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStrea
     const size_t S = size_t(32) * f.lw, Vs = size_t(kFrontThreads) * f.rpt;
     const size_t smem = S * 4 + Vs * 4 + S * 2;
     cudaError_t e;
-    if (index_type == DST_I64) {
+    if (index_type == DST_I64)
         e = cudaFuncSetAttribute(k_front_cluster<long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        return launch_pdl(k_front_cluster<long long>, dim3(grid), dim3(kFrontThreads), smem, stream, f);
-    } else {
+    else
         e = cudaFuncSetAttribute(k_front_cluster<int>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        return launch_pdl(k_front_cluster<int>, dim3(grid), dim3(kFrontThreads), smem, stream, f);
+    if (e != cudaSuccess) return e;
+    // Copy clusters: no more than can be resident beside the index cluster (a cluster needs eight free SMs of
+    // one GPC; clusters that start late would finish late, their share of the rows being fixed).
+    int copy_clusters = p.copy_clusters > 0 ? p.copy_clusters : 0;
+    if (copy_clusters > 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kClusterCtas * (1 + copy_clusters)); cfg.blockDim = dim3(kFrontThreads); cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kClusterCtas; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        // the answer depends on the device and on the shared memory asked for: remembered per index type
+        static std::atomic<long long> cache[2];
+        const int which = index_type == DST_I64 ? 1 : 0;
+        int dev = 0;
+        (void)cudaGetDevice(&dev);
+        const long long key = ((long long)smem << 16) | ((long long)(dev & 0xFF) << 8);
+        const long long seen = cache[which].load();
+        int resident = 0;
+        if ((seen & ~0xFFLL) == key && (seen & 0xFF) != 0) {
+            resident = int(seen & 0xFF);
+        } else {
+            if (which) e = cudaOccupancyMaxActiveClusters(&resident, k_front_cluster<long long>, &cfg);
+            else e = cudaOccupancyMaxActiveClusters(&resident, k_front_cluster<int>, &cfg);
+            if (e != cudaSuccess) { (void)cudaGetLastError(); resident = 0; }
+            if (resident > 0) cache[which].store(key | (resident > 255 ? 255 : resident));
+        }
+        if (resident >= 2 && copy_clusters > resident - 1) copy_clusters = resident - 1;
     }
-    return cudaGetLastError();
+    const int grid = kClusterCtas * (1 + copy_clusters);
+    if (index_type == DST_I64)
+        return launch_pdl(k_front_cluster<long long>, dim3(grid), dim3(kFrontThreads), smem, stream, f);
+    return launch_pdl(k_front_cluster<int>, dim3(grid), dim3(kFrontThreads), smem, stream, f);
 }
 
 }  // namespace dst

@@ -422,13 +422,18 @@ struct WarpPipe {
     // A batch of consecutive output rows: their entries and their closing units, flattened
     __device__ bool do_rows(int batch, int cblk) {
         const int2 bt = a.batches[batch];
-        if (bt.x == 0) return true;                       // no row starts in this batch
-        const int v0 = bt.x - 1;
+        if (bt.y == 0) return true;                       // no row starts in this batch
+        const int v0 = bt.x - 1;                          // first row (compact: its rank among the named rows)
         const int nrows = min(bt.y - bt.x + 1, 31);
         const long long cb = (long long)cblk * a.W;
         const long long wcols = min((long long)a.W, a.d - cb);
-        int o = 0;
-        if (lane <= nrows) o = a.offsets[v0 + lane];
+        int o = 0, row = v0 + lane;
+        if (a.compact) {
+            if (lane <= nrows) o = a.uoff[v0 + lane];
+            if (lane < nrows) row = a.urow[v0 + lane];
+        } else {
+            if (lane <= nrows) o = a.offsets[v0 + lane];
+        }
         const int o_next = __shfl_down_sync(0xFFFFFFFFu, o, 1);
         const int cnt = lane < nrows ? o_next - o : 0;
         const int nunits = (lane < nrows && cnt <= a.chunk) ? cnt + 1 : 0;   // heavy rows belong to the chunk items
@@ -452,7 +457,8 @@ struct WarpPipe {
             const int e = q - (__shfl_sync(0xFFFFFFFFu, incl, i) - __shfl_sync(0xFFFFFFFFu, nunits, i));
             const int ci = __shfl_sync(0xFFFFFFFFu, cnt, i);
             const int oi = __shfl_sync(0xFFFFFFFFu, o, i);
-            UnitBlock b{nullptr, 0u, 0, 0};
+            const int vi = __shfl_sync(0xFFFFFFFFu, row, i);
+            UnitBlock b{nullptr, 0u, 0, vi};
             if (q < total) {
                 if (e < ci) {
                     const unsigned p = a.perm[oi + e];
@@ -462,11 +468,8 @@ struct WarpPipe {
                         b.kind = kUnitAdd;
                     }
                 } else {
-                    b.y = v0 + i;
                     b.kind = kUnitFinal | (ci == 0 ? kUnitCopy : 0);
-                    if (ci == 0 && b.y < a.precopied) {
-                        b.kind = 0;                       // the row already holds its dense_in row (or zeros)
-                    } else if (a.dense_in) {
+                    if (a.dense_in) {
                         b.src = static_cast<const OT*>(a.dense_in) + (long long)b.y * a.d + cb;
                         b.bytes = (unsigned)(wcols * (long long)sizeof(OT));
                     }
@@ -606,15 +609,6 @@ static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaSt
     const PipeShape ps = pipe_shape((int)sizeof(VT), (int)sizeof(OT), a.d);
     a.W = ps.W; a.ncb = ps.ncb; a.slot_bytes = ps.slot_bytes; a.n_slots = ps.n_slots;
     int ctas_per_sm = ps.ctas_per_sm;
-    if (false && a.precopied && a.n_slots > 3) {
-        // Pre-filled output: few bytes left to move, bound by the latency of a work item: shallower rings,
-        // more warps.
-        a.n_slots = 3;
-        const int per_cta = kPipeHeaderReserve + kPipeWarps * a.n_slots * ps.slot_bytes + 1024 + 256;
-        ctas_per_sm = kSmemPerSm / per_cta;
-        if (ctas_per_sm > 3) ctas_per_sm = 3;      // what the kernel's registers allow
-        if (ctas_per_sm < ps.ctas_per_sm) ctas_per_sm = ps.ctas_per_sm;
-    }
     const size_t smem = size_t(kPipeHeaderReserve) + size_t(kPipeWarps) * size_t(a.n_slots) * size_t(ps.slot_bytes);
     const int grid = sm_count * ctas_per_sm;
     constexpr int kMaxK = sizeof(VT) == 4 ? 8 : 4;
