@@ -21,7 +21,7 @@ constexpr int kFrontMaxRows = 65535;        // largest input (positions are pack
 constexpr int kPrepItems = 8;               // indices per thread of the validation kernel
 constexpr int kPrepTile = kSortThreads * kPrepItems;
 constexpr int kMaxPasses = 4;               // 8-bit digits, keys below 2^31
-constexpr int kFanIn = 16;                  // children per node of the heavy-row combine tree
+constexpr int kFanIn = 8;                   // children per node of the heavy-row combine tree
 constexpr int kMaxBatchUnits = 31;          // a light work item holds rows worth at most this many units (+ one row)
 constexpr int kMaxChunkBytes = 256 * 1024;  // value bytes per chunk of a heavy row (at most): 64 fp32 rows of 1024 columns
 constexpr int kPipeWarpsTotal = 148 * 8;    // warps the row-reduction kernel runs with on a B200 (sizes the work items)
