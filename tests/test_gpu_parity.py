@@ -7,7 +7,7 @@ import oracle
 import paper_1905_04035_b200 as dst
 from paper_1905_04035_b200.workloads import Workload, make_workload, to_bf16_bits
 
-from gpu_helpers import assert_parity, oracle_of, raw_bits, run_library, to_numpy_f64
+from gpu_helpers import assert_parity, oracle_of, raw_bits, run_library, to_device, to_numpy_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -230,6 +230,29 @@ def test_prefilled_output_bf16_and_out_of_range():
     assert_parity(w, run_library(w))
     w = _custom(vocab, 256, [4000], idx_fn=idx, value_dtype="bf16", out_dtype="f32", with_dense=False)
     assert_parity(w, run_library(w))
+
+
+@pytest.mark.parametrize("name,scale", [("big", 1.0), ("r64", 0.1)])
+def test_cuda_graph_replay_matches_eager_calls(name, scale):
+    # the benchmark times CUDA-graph replays of one library call: same bits as the eager call, replay after replay
+    w = make_workload(name, scale=scale)
+    eager = run_library(w, mode="concat")
+    assert_parity(w, eager)
+    slices = [(to_device(i, w.index_dtype), to_device(v, w.value_dtype)) for i, v in zip(w.indices, w.values)]
+    dense = to_device(w.dense_in, w.out_dtype)
+    out = torch.full((w.vocab, w.d), float("nan"), device="cuda")
+    eng = dst.Densifier(w.n_rows_total, w.R, w.d, w.vocab)
+    eng(slices, dense, out)                        # first call outside capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        eng(slices, dense, out)
+    for _ in range(3):
+        out.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(raw_bits(out), raw_bits(eager.out))
+        assert eng.read_result()["status"] == 0 and eng.read_result()["n_unique"] == eager.result["n_unique"]
 
 
 def test_many_slices_use_several_histogram_launches():
