@@ -316,14 +316,26 @@ struct WarpPipe {
             const bool root = n_parent == 1;
             sum_children(acc, child_first + parent * kFanIn, n_children, cb, wcols);
             if (root) {
+                // The output may be the dense input itself, so the compiler keeps loads and stores in
+                // program order: read the whole dense row first, then store, or every column group
+                // pays its own trip to memory.
                 const OT* din = static_cast<const OT*>(a.dense_in);
                 OT* out = static_cast<OT*>(a.out) + (long long)hi.row * a.d + cb;
+                constexpr int KH = (sizeof(VT) == 2 && K >= 4) ? K / 2 : K;
 #pragma unroll
-                for (int k = 0; k < K; ++k) {
-                    const int c = col(k);
-                    if (c < wcols) {
-                        if (din) { Acc<VC> dn; load_elems(din + (long long)hi.row * a.d + cb + c, dn); add(acc[k], dn); }
-                        store_out(out + c, acc[k]);
+                for (int h0 = 0; h0 < K; h0 += KH) {
+                    Acc<VC> dn[KH];
+#pragma unroll
+                    for (int k = 0; k < KH; ++k) {
+                        const int c = col(h0 + k);
+                        zero(dn[k]);
+                        if (din && c < wcols) load_elems(din + (long long)hi.row * a.d + cb + c, dn[k]);
+                    }
+#pragma unroll
+                    for (int k = 0; k < KH; ++k) {
+                        const int c = col(h0 + k);
+                        add(acc[h0 + k], dn[k]);
+                        if (c < wcols) store_out(out + c, acc[h0 + k]);
                     }
                 }
                 return;
@@ -374,16 +386,18 @@ struct WarpPipe {
             }
             if (kind & kUnitFinal) {
                 OT* orow = out + (long long)y * a.d + cb;
+                Acc<VC> dn[K];                            // the dense row first, all of it, then the stores
 #pragma unroll
                 for (int k = 0; k < K; ++k) {
                     const int c = col(k);
-                    if (c < wcols) {
-                        Acc<VC> dn;
-                        zero(dn);
-                        if (a.dense_in) load_elems(reinterpret_cast<const OT*>(sp) + c, dn);
-                        if (!(kind & kUnitCopy)) add(dn, acc[k]);
-                        store_out(orow + c, dn);
-                    }
+                    zero(dn[k]);
+                    if (a.dense_in && c < wcols) load_elems(reinterpret_cast<const OT*>(sp) + c, dn[k]);
+                }
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const int c = col(k);
+                    if (!(kind & kUnitCopy)) add(dn[k], acc[k]);
+                    if (c < wcols) store_out(orow + c, dn[k]);
                     zero(acc[k]);
                 }
             }
