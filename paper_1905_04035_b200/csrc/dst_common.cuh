@@ -27,10 +27,9 @@ constexpr int kMaxChunkBytes = 256 * 1024;  // value bytes per chunk of a heavy 
 constexpr int kPipeWarpsTotal = 148 * 8;    // warps the row-reduction kernel runs with on a B200 (sizes the work items)
 constexpr int kPipeWarps = 4;               // row-reduction kernel: warps per CTA, each with its own slot ring
 constexpr int kPipeThreads = kPipeWarps * 32;
-constexpr int kPipeSlots = 6;               // ring slots per warp
+constexpr int kPipeSlots = 6;               // ring slots per warp, at most
 constexpr int kPipeHeaderReserve = 1024;    // mbarriers in front of the slots
 constexpr int kMaxBlockCols = 1024;         // columns per column block (32 fp32 accumulators per lane)
-constexpr int kSmemPerSm = 227 * 1024;
 constexpr long long kWaitCycles = 1LL << 31; // SM clock cycles (about a second) before an mbarrier wait gives up
 constexpr int kScanThreads = 256;
 constexpr int kScanItems = 8;               // rows per thread in the scan kernel
@@ -133,7 +132,7 @@ struct MainArgs {
 };
 
 // How the row-reduction kernel cuts rows into column blocks and shared memory into slots.
-struct PipeShape { int K, W, ncb, slot_bytes, n_slots, ctas_per_sm; };
+struct PipeShape { int K, W, ncb, slot_bytes, n_slots; };
 inline PipeShape pipe_shape(int value_size, int out_size, int64_t d) {
     PipeShape p{};
     const int vc = 16 / value_size;                        // columns per 16-byte group of a value row
@@ -144,10 +143,7 @@ inline PipeShape pipe_shape(int value_size, int out_size, int64_t d) {
     while (p.K * 32 * vc < p.W) p.K *= 2;                  // 16-byte groups per lane
     const int widest = value_size > out_size ? value_size : out_size;
     p.slot_bytes = (p.W * widest + 127) / 128 * 128;
-    p.n_slots = kPipeSlots;
-    const int per_cta = kPipeHeaderReserve + kPipeWarps * p.n_slots * p.slot_bytes + 1024 + 5376;   // + the driver's reserve + the kernel's static tables
-    int c = kSmemPerSm / per_cta;
-    p.ctas_per_sm = c < 1 ? 1 : (c > 8 ? 8 : c);
+    p.n_slots = kPipeSlots;                                // at most; the launcher may use fewer
     return p;
 }
 

@@ -227,9 +227,57 @@ struct WarpPipe {
 
     __device__ __forceinline__ float* partial_row(int slot) const { return a.partials + (long long)slot * a.d; }
 
-    // acc = child[0] + child[1] + ... in index order (bf16: half of the column groups at a time, to save registers)
-    __device__ __forceinline__ void sum_children(Acc<VC> (&acc)[K], int first_slot, int n, long long cb, int wcols) const {
+    // a plain copy of `bytes` bytes into the next slot (lane 0 talks to the copy engine)
+    __device__ __forceinline__ void issue_plain(const void* src, unsigned bytes) {
+        if (lane == 0) {
+            const unsigned bar = bars + 8u * (unsigned)islot;
+            mbar_arrive_expect_tx(bar, bytes);
+            bulk_load(ring + (unsigned)islot * (unsigned)a.slot_bytes, src, bytes, bar);
+        }
+        issued_mask |= 1u << islot;
+        islot = islot + 1 == a.n_slots ? 0 : islot + 1;
+    }
+
+    // acc = child[0] + child[1] + ... in index order.  fp32 value rows: a slot of the ring holds one
+    // partial row, so the children stream through the ring like any other unit, n_slots copies in
+    // flight, and the sum costs about one trip to memory however busy the memory system is.
+    // bf16 value rows (slots half as wide as a partial row): direct loads, half of the column
+    // groups at a time to save registers.
+    // `last_row`, when given, is one more fp32 row added after the children (the dense row at the root).
+    __device__ __forceinline__ bool sum_children(Acc<VC> (&acc)[K], int first_slot, int n_children, long long cb, int wcols,
+                                                 const float* last_row) {
+        if constexpr (sizeof(VT) == 4) {
+            const int n = n_children + (last_row ? 1 : 0);
+            auto source = [&](int c) { return c < n_children ? partial_row(first_slot + c) + cb : last_row; };
+            // the partial rows were written with ordinary stores; the copy engine reads them
+            asm volatile("fence.proxy.async;" ::: "memory");
+#pragma unroll
+            for (int k = 0; k < K; ++k) zero(acc[k]);
+            const unsigned bytes = (unsigned)wcols * 4u;
+            int issued = 0;
+            for (; issued < n && issued < a.n_slots; ++issued) issue_plain(source(issued), bytes);
+            for (int c = 0; c < n; ++c) {
+                if (!mbar_wait(bars + 8u * (unsigned)cslot, (cphase >> cslot) & 1u, abort_flag)) { give_up(); return false; }
+                cphase ^= 1u << cslot;
+                issued_mask &= ~(1u << cslot);
+                const VT* sp = reinterpret_cast<const VT*>(ring_ptr + (size_t)cslot * a.slot_bytes);
+                Acc<VC> v[K];
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const int cc = col(k);
+                    zero(v[k]);
+                    if (cc < wcols) load_elems(sp + cc, v[k]);
+                }
+#pragma unroll
+                for (int k = 0; k < K; ++k) add(acc[k], v[k]);
+                __syncwarp();
+                cslot = cslot + 1 == a.n_slots ? 0 : cslot + 1;
+                if (issued < n) { issue_plain(source(issued), bytes); ++issued; }
+            }
+            return true;
+        }
         constexpr int KH = (sizeof(VT) == 2 && K >= 4) ? K / 2 : K;   // the bf16 variants run at 128 registers
+        const int n = n_children;
 #pragma unroll
         for (int h0 = 0; h0 < K; h0 += KH) {
 #pragma unroll
@@ -251,6 +299,7 @@ struct WarpPipe {
                 for (int k = 0; k < KH; ++k) { add(acc[h0 + k], va[k]); add(acc[h0 + k], vb[k]); }
             }
         }
+        return true;
     }
 
     // Heavy row that owns chunk cid: the last h with heavy[h].chunk_base <= cid.
@@ -284,7 +333,7 @@ struct WarpPipe {
 
     // The chunk's sum is in acc: store it as a partial row and climb the combine tree while this
     // warp is the last child to arrive.
-    __device__ void finish_chunk(Acc<VC> (&acc)[K], int cid, int cblk) const {
+    __device__ bool finish_chunk(Acc<VC> (&acc)[K], int cid, int cblk) {
         const HeavyInfo hi = cur_heavy;
         const long long cb = (long long)cblk * a.W;
         const int wcols = (int)min((long long)a.W, a.d - cb);
@@ -311,15 +360,20 @@ struct WarpPipe {
             int last = 0;
             if (lane == 0) last = atomicAdd(&node_cnt[node], 1u) == (unsigned)(n_children - 1);
             last = __shfl_sync(0xFFFFFFFFu, last, 0);
-            if (!last) return;
+            if (!last) return true;
             __threadfence();
             const bool root = n_parent == 1;
-            sum_children(acc, child_first + parent * kFanIn, n_children, cb, wcols);
+            // fp32 rows in, fp32 rows out: the root's dense row rides the ring behind the children
+            constexpr bool kDenseInRing = sizeof(VT) == 4 && sizeof(OT) == 4;
+            const float* dense_row = nullptr;
+            if constexpr (kDenseInRing)
+                if (root && a.dense_in) dense_row = static_cast<const float*>(a.dense_in) + (long long)hi.row * a.d + cb;
+            if (!sum_children(acc, child_first + parent * kFanIn, n_children, cb, wcols, dense_row)) return false;
             if (root) {
                 // The output may be the dense input itself, so the compiler keeps loads and stores in
                 // program order: read the whole dense row first, then store, or every column group
                 // pays its own trip to memory.
-                const OT* din = static_cast<const OT*>(a.dense_in);
+                const OT* din = kDenseInRing ? nullptr : static_cast<const OT*>(a.dense_in);
                 OT* out = static_cast<OT*>(a.out) + (long long)hi.row * a.d + cb;
                 constexpr int KH = (sizeof(VT) == 2 && K >= 4) ? K / 2 : K;
 #pragma unroll
@@ -338,7 +392,7 @@ struct WarpPipe {
                         if (c < wcols) store_out(out + c, acc[h0 + k]);
                     }
                 }
-                return;
+                return true;
             }
             float* pr = partial_row(a.chunk_max + node) + cb;
 #pragma unroll
@@ -405,7 +459,7 @@ struct WarpPipe {
             cslot = cslot + 1 == a.n_slots ? 0 : cslot + 1;
             if (j + a.n_slots < n) issue(b, j + a.n_slots);   // refill it
             if (kind & kUnitChunkEnd) {
-                finish_chunk(acc, y, cblk);
+                if (!finish_chunk(acc, y, cblk)) return false;
 #pragma unroll
                 for (int k = 0; k < K; ++k) zero(acc[k]);
             }
@@ -603,11 +657,25 @@ k_reduce_rows_scalar(const MainArgs a) {
     }
 }
 
+// Copies kept in flight by the whole grid.  Enough to cover the memory system's latency at full
+// bandwidth with some slack; more only lengthens the queue every dependent access waits in (an
+// index lookup, a node of a combine tree), which is what a short call is made of.
+constexpr long long kInFlightBytes = 14ll << 20;
+
 template <typename VT, typename OT, int K>
-static cudaError_t launch_pipe(const MainArgs& a, int grid, size_t smem, cudaStream_t stream) {
-    cudaError_t e = cudaFuncSetAttribute(k_reduce_rows<VT, OT, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+static cudaError_t launch_pipe(MainArgs a, int sm_count, cudaStream_t stream) {
+    auto smem_for = [&](int slots) { return size_t(kPipeHeaderReserve) + size_t(kPipeWarps) * size_t(slots) * size_t(a.slot_bytes); };
+    cudaError_t e = cudaFuncSetAttribute(k_reduce_rows<VT, OT, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_for(kPipeSlots));
     if (e != cudaSuccess) return e;
-    return launch_pdl(k_reduce_rows<VT, OT, K>, dim3(grid), dim3(kPipeThreads), smem, stream, a);
+    int resident = 0;                                    // CTAs of this variant an SM holds with full rings
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, k_reduce_rows<VT, OT, K>, kPipeThreads, smem_for(kPipeSlots));
+    if (e != cudaSuccess) return e;
+    if (resident < 1) return cudaErrorLaunchOutOfResources;
+    const int grid = sm_count * resident;
+    const long long per_slot = (long long)grid * kPipeWarps * a.slot_bytes;
+    long long slots = kInFlightBytes / per_slot;
+    a.n_slots = (int)(slots < 2 ? 2 : (slots > kPipeSlots ? kPipeSlots : slots));
+    return launch_pdl(k_reduce_rows<VT, OT, K>, dim3(grid), dim3(kPipeThreads), smem_for(a.n_slots), stream, a);
 }
 
 template <typename VT, typename OT>
@@ -622,14 +690,11 @@ static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaSt
     }
     const PipeShape ps = pipe_shape((int)sizeof(VT), (int)sizeof(OT), a.d);
     a.W = ps.W; a.ncb = ps.ncb; a.slot_bytes = ps.slot_bytes; a.n_slots = ps.n_slots;
-    int ctas_per_sm = ps.ctas_per_sm;
-    const size_t smem = size_t(kPipeHeaderReserve) + size_t(kPipeWarps) * size_t(a.n_slots) * size_t(ps.slot_bytes);
-    const int grid = sm_count * ctas_per_sm;
     constexpr int kMaxK = sizeof(VT) == 4 ? 8 : 4;
-    if (ps.K == 1) return launch_pipe<VT, OT, 1>(a, grid, smem, stream);
-    if (ps.K == 2) return launch_pipe<VT, OT, 2>(a, grid, smem, stream);
-    if (ps.K == 4 || kMaxK == 4) return launch_pipe<VT, OT, 4>(a, grid, smem, stream);
-    return launch_pipe<VT, OT, kMaxK>(a, grid, smem, stream);
+    if (ps.K == 1) return launch_pipe<VT, OT, 1>(a, sm_count, stream);
+    if (ps.K == 2) return launch_pipe<VT, OT, 2>(a, sm_count, stream);
+    if (ps.K == 4 || kMaxK == 4) return launch_pipe<VT, OT, 4>(a, sm_count, stream);
+    return launch_pipe<VT, OT, kMaxK>(a, sm_count, stream);
 }
 
 cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,
