@@ -23,7 +23,7 @@ constexpr int kPrepTile = kSortThreads * kPrepItems;
 constexpr int kMaxPasses = 4;               // 8-bit digits, keys below 2^31
 constexpr int kFanIn = 8;                   // children per node of the heavy-row combine tree
 constexpr int kMaxBatchUnits = 31;          // a light work item holds rows worth at most this many units (+ one row)
-constexpr int kMaxChunkBytes = 256 * 1024;  // value bytes per chunk of a heavy row (at most): 64 fp32 rows of 1024 columns
+constexpr int kMaxChunkRows = 128;           // entries per chunk of a heavy row, at most (fewer chunks mean fewer drains of a warp's ring; more make the last items too long)
 constexpr int kPipeWarpsTotal = 148 * 8;    // warps the row-reduction kernel runs with on a B200 (sizes the work items)
 constexpr int kPipeWarps = 4;               // row-reduction kernel: warps per CTA, each with its own slot ring
 constexpr int kPipeThreads = kPipeWarps * 32;
@@ -158,9 +158,7 @@ inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab, i
     // so that the tail of the row-reduction kernel stays short.
     const int64_t share = (vocab + n_rows) / (int64_t(kPipeWarpsTotal) * 3);
     int c = 16;
-    int64_t row_bytes = (d < kMaxBlockCols ? d : kMaxBlockCols) * int64_t(value_size);
-    if (row_bytes < 1) row_bytes = 1;
-    const int64_t max_chunk = kMaxChunkBytes / row_bytes < 64 ? 64 : (kMaxChunkBytes / row_bytes > 256 ? 256 : kMaxChunkBytes / row_bytes);
+    const int64_t max_chunk = kMaxChunkRows;
     while (c < max_chunk && c * 2 <= share) c *= 2;
     L.batch_units = int(share < 8 ? 8 : (share > kMaxBatchUnits ? kMaxBatchUnits : share));
     L.batch_max = (vocab + n_rows) / L.batch_units + 2;

@@ -39,12 +39,18 @@ k_prep(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, unsigne
     const IT* __restrict__ idx = static_cast<const IT*>(se.indices);
     const int lane = lane_id();
     unsigned bad = 0;
+    long long vals[kPrepItems];          // every index of this thread first: one trip to memory, not kPrepItems
+#pragma unroll
+    for (int k = 0; k < kPrepItems; ++k) {
+        const long long i = t0 + k * kSortThreads + threadIdx.x;
+        vals[k] = -1;
+        if (i < n) vals[k] = (long long)idx[i];
+    }
 #pragma unroll
     for (int k = 0; k < kPrepItems; ++k) {
         const long long i = t0 + k * kSortThreads + threadIdx.x;
         const bool in = i < n;
-        long long v = -1;
-        if (in) v = (long long)idx[i];
+        const long long v = vals[k];
         const bool ok = in && v >= 0 && v < vocab;
         const unsigned key = ok ? (unsigned)v : kInvalidKey;
         if (in) keys[se.start + i] = key;
@@ -111,12 +117,15 @@ k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, c
     pdl_trigger();
     pdl_wait();
     if (threadIdx.x == 0) s_tile = atomicAdd(&hdr->ticket[pass], 1u);   // tiles start in id order
+    // asked for now, needed later: these two trips to memory overlap the ticket's
+    const unsigned n_bad = pass == 0 ? 0u : (unsigned)hdr->n_bad;
+    const unsigned g = digit_hist[threadIdx.x];   // kSortThreads == 256 digits
     for (int s = threadIdx.x; s < kWarps * 256; s += kSortThreads) (&wh[0][0])[s] = 0;
     __syncthreads();
     const int tile = (int)s_tile;
     // pass 0 reads every input position (invalid rows carry kInvalidKey and drop out);
     // later passes read the survivors
-    const int n_in = pass == 0 ? capacity : capacity - (int)hdr->n_bad;
+    const int n_in = capacity - (int)n_bad;
     const long long t0 = (long long)tile * kTile;
     if (t0 >= n_in) return;
 
@@ -153,7 +162,6 @@ k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, c
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) { unsigned t = wh[w][d]; wh[w][d] = cnt; cnt += t; }
     // where digit d starts globally: exclusive scan of this pass's digit histogram
-    unsigned g = digit_hist[d];
     unsigned ginc = g;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { unsigned t = __shfl_up_sync(0xFFFFFFFFu, ginc, o); if (lane >= o) ginc += t; }
