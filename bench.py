@@ -259,6 +259,26 @@ def time_device_graph(prob: DeviceProblem, steps: int, warmup: int, dist_ctx=Non
     return total_ms, clock_info
 
 
+def time_device_warm(prob: DeviceProblem, steps: int, warmup: int):
+    """The warm figure beside the cold one: the same call replayed on ONE buffer set with no flush, so
+    whatever part of the inputs fits in L2 is still there.  Returns ms per step."""
+    import torch
+    slices, dense, out = prob.sets[0]
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        prob.eng(slices, dense, out)
+    for _ in range(warmup):
+        g.replay()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for _ in range(steps):
+        g.replay()
+    t1.record()
+    torch.cuda.synchronize()
+    return t0.elapsed_time(t1) / steps
+
+
 def time_e2e(w, device, steps: int, warmup: int):
     """Same metric through the host entry point: pinned host buffers, H2D and D2H inside the timed region."""
     import torch
@@ -297,8 +317,11 @@ def time_e2e(w, device, steps: int, warmup: int):
 # ---------------------------------------------------------------------------------------------
 # the CPU oracle arm (reference arm and cpu_baseline leg)
 # ---------------------------------------------------------------------------------------------
-def time_oracle(w, max_rows=None, repeats=1):
-    """Time the oracle as it stands on (a prefix of every slice of) the workload.  Single thread."""
+def time_oracle(w, max_rows=None, repeats=1, threads=False):
+    """Time the oracle as it stands on (a prefix of every slice of) the workload.  Single thread.
+
+    ``threads=True`` times the other CPU baseline instead: the same loop in fp32, one thread per
+    block of columns, on every core this process may use."""
     import oracle
     idx, val = w.indices, w.values
     sample = "full workload"
@@ -310,15 +333,21 @@ def time_oracle(w, max_rows=None, repeats=1):
             keep, w.R, keep * w.R, w.n_rows_total)
     n = int(sum(i.shape[0] for i in idx))
     best = None
+    cores = 1
     for _ in range(repeats):
         t = time.perf_counter()
-        oracle.densify(idx, val, w.d, w.vocab, w.dense_in, value_dtype=w.value_dtype, out_dtype=w.out_dtype)
+        if threads:
+            cores = oracle.densify_threads(idx, val, w.d, w.vocab, w.dense_in, value_dtype=w.value_dtype,
+                                           out_dtype=w.out_dtype)[2]
+        else:
+            oracle.densify(idx, val, w.d, w.vocab, w.dense_in, value_dtype=w.value_dtype, out_dtype=w.out_dtype)
         dt = time.perf_counter() - t
         best = dt if best is None else min(best, dt)
     b = n * w.d * SIZEOF[w.value_dtype] + w.vocab * w.d * SIZEOF[w.out_dtype] + n * SIZEOF[w.index_dtype]
     if w.dense_in is not None:
         b += w.vocab * w.d * SIZEOF[w.out_dtype]
-    return {"seconds": best, "rows": n, "bytes": b, "gbs": b / best / 1e9, "rows_per_s": n / best, "sample": sample}
+    return {"seconds": best, "rows": n, "bytes": b, "gbs": b / best / 1e9, "rows_per_s": n / best, "sample": sample,
+            "cores": cores}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -336,6 +365,7 @@ def run_config(name, device, steps, warmup, seed, dist_ctx=None, clocks=None, wa
     else:
         total_ms, _, _, clock_info = time_device(prob, steps, warmup, dist_ctx, clocks)
     ms = total_ms / steps
+    warm_ms = time_device_warm(prob, steps, warmup) if use_graph and dist_ctx is None else None
     kms = float(np.mean(kernel_ms))
     # small inputs: part of the output is filled by the index kernel's extra clusters, so the row-reduction
     # kernel does not move all of the step's bytes and has no roofline figure of its own
@@ -345,7 +375,7 @@ def run_config(name, device, steps, warmup, seed, dist_ctx=None, clocks=None, wa
         "frac_of_hbm_peak": prob.balg / ms / 1e6 / peak, "algorithmic_bytes": prob.balg,
         "reduce_kernel_ms": kms, "reduce_kernel_gbs": None if prefilled else prob.balg / kms / 1e6,
         "reduce_kernel_frac": None if prefilled else prob.balg / kms / 1e6 / peak, "launches": launches, "l2": prob.l2_policy(),
-        "eager_ms_per_step": eager_ms / steps, "cuda_graph": bool(use_graph),
+        "eager_ms_per_step": eager_ms / steps, "warm_ms_per_step": warm_ms, "cuda_graph": bool(use_graph),
         "n_unique": res["n_unique"], "max_segment": res["max_segment"], "status": res["status"],
         "peak_gbs": peak, "peak_source": peak_src, "clocks": clock_info, "w": w,
     }
@@ -450,14 +480,18 @@ def main():
             r = run_config(name, device, min(args.steps, 200), args.warmup, args.seed, use_graph=not args.no_graph)
             r.pop("w"); r.pop("clocks")
             others.append({k: r[k] for k in ("workload", "ms_per_step", "gbs", "rows_per_s", "frac_of_hbm_peak",
-                                             "algorithmic_bytes", "reduce_kernel_ms", "reduce_kernel_frac", "l2", "eager_ms_per_step",
+                                             "algorithmic_bytes", "reduce_kernel_ms", "reduce_kernel_frac", "l2", "eager_ms_per_step", "warm_ms_per_step",
                                              "n_unique", "max_segment", "status")})
 
-    cpu = None
+    cpu = cpu_threads = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         info = time_oracle(w, max_rows=None if w.n_rows_total <= 700000 else 700000)
         cpu = {"value": info["gbs"], "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": info["sample"],
                "seconds": info["seconds"], "rows_per_s": info["rows_per_s"]}
+        info = time_oracle(w, max_rows=None if w.n_rows_total <= 700000 else 700000, repeats=2, threads=True)
+        cpu_threads = {"value": info["gbs"], "unit": "GB/s", "cores": info["cores"],
+                       "kind": "fp32 loop, one thread per block of columns", "sample": info["sample"],
+                       "seconds": info["seconds"], "rows_per_s": info["rows_per_s"]}
 
     if rank == 0:
         rep = dst.dst_bytes_report([int(i.shape[0]) for i in w.indices], w.d, w.vocab,
@@ -472,7 +506,7 @@ def main():
                        "n_rows_total": w.n_rows_total, "l2": head["l2"], "replicas": world, "scale": args.scale,
                        "timed_as": "CUDA-graph replay of one library call per step" if head["cuda_graph"]
                        else "eager library calls"},
-            "eager_ms_per_step": head["eager_ms_per_step"],
+            "eager_ms_per_step": head["eager_ms_per_step"], "warm_ms_per_step": head["warm_ms_per_step"],
             "rows_per_s": agg["rows_per_s"], "frac_of_hbm_peak": agg["gbs"] / world / head["peak_gbs"],
             "roofline": {"bound": "hbm", "achieved": head["reduce_kernel_gbs"], "peak": head["peak_gbs"],
                          "unit": "GB/s", "frac": head["reduce_kernel_frac"],
@@ -480,7 +514,7 @@ def main():
                          "kernel": "k_reduce_rows", "of": head["peak_source"],
                          "kernel_ms": head["reduce_kernel_ms"]},
             "e2e": e2e, "gpu_launches": head["launches"], "clocks": head["clocks"],
-            "cpu_baseline": cpu, "bytes_report": rep, "all_configs": others,
+            "cpu_baseline": cpu, "cpu_baseline_threads": cpu_threads, "bytes_report": rep, "all_configs": others,
             "parity": {"status": head["status"], "n_unique": head["n_unique"], "max_segment": head["max_segment"]},
         }
         print(json.dumps(line))

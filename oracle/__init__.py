@@ -7,3 +7,4 @@ from .dst_oracle import (  # noqa: F401
     round_bf16,
     widen_bf16,
 )
+from .cpu_threads import build_cpu_threads_library, densify_threads, host_cores  # noqa: F401,E402
