@@ -179,6 +179,75 @@ int dst_densify_concat_host(const dst_slice_t* slices, int32_t R, int64_t d, int
                             void* workspace, size_t workspace_bytes, dst_result_t* host_result);
 
 /*
+ * Accumulating a list of gradients of one variable: the strategies of the paper.
+ *
+ * A gradient is either a dense [vocab, d] tensor (DST_GRAD_DENSE: `values` holds it, in
+ * opts->out_type; `indices` and `n_rows` are ignored) or IndexedSlices (DST_GRAD_SLICES:
+ * `indices` [n_rows] in opts->index_type, `values` [n_rows, d] in opts->value_type).
+ *
+ *   DST_ACC_STOCK            Algorithm 1 (Section 3): fewer than two gradients pass through; if all
+ *                            are dense they are summed ("reduce"); otherwise every gradient is
+ *                            treated as IndexedSlices -- a dense one becomes vocab slices, row v
+ *                            with index v -- and they are concatenated in the order given ("gather").
+ *   DST_ACC_PROPOSED         Algorithm 2 (Section 6): as above, but if at least one gradient is dense
+ *                            every gradient is converted to a dense tensor and they are summed.
+ *   DST_ACC_SPARSE_AS_DENSE  Listing 1 (Section 4): every IndexedSlices gradient is converted to a
+ *                            dense tensor first, then Algorithm 1 runs (and can only reduce).
+ *
+ * dst_accumulate_plan (host only, touches no device memory) says which branch a list takes, what
+ * the output is and how large: call it to size the output buffers and the workspace
+ * (dst_workspace_bytes(plan.n_slice_rows, plan.n_slices, d, vocab, opts) when plan.converts != 0).
+ *
+ * dst_accumulate enqueues the work on `stream`:
+ *   - dense output  -> out_dense [vocab, d] in opts->out_type.  The dense gradients are added left to
+ *     right in fp32, then the slices are densified onto that sum in one pass (dst_densify_concat
+ *     with out_dense as its dense partner), so the value rows cross the memory bus once.
+ *     `result` (optional) is written only when slices were converted (plan.converts != 0).
+ *   - slices output -> out_indices [out_rows], out_values [out_rows, d]: the concatenation.  Needs
+ *     out_capacity_rows >= plan.out_rows, and value_type == out_type when a dense gradient is
+ *     among them (its rows are copied, not converted); otherwise DST_ERR_UNSUPPORTED.
+ *   - an empty list enqueues nothing (plan.out_kind == -1).
+ * A pass-through copies the one gradient into the output buffers of its kind.  `grads` is a HOST
+ * array read during the call only.  Outputs must not overlap inputs, except that out_dense may be
+ * one of the dense gradients.  `plan` (optional, host) receives what dst_accumulate_plan returns.
+ */
+typedef enum { DST_GRAD_DENSE = 0, DST_GRAD_SLICES = 1 } dst_grad_kind_t;
+typedef struct {
+    int32_t kind; /* dst_grad_kind_t */
+    int32_t reserved;
+    const void* indices;
+    const void* values;
+    int64_t n_rows;
+} dst_grad_t;
+typedef enum { DST_ACC_STOCK = 0, DST_ACC_PROPOSED = 1, DST_ACC_SPARSE_AS_DENSE = 2 } dst_strategy_t;
+typedef enum {
+    DST_BRANCH_EMPTY = 0,
+    DST_BRANCH_PASS_THROUGH = 1,
+    DST_BRANCH_REDUCE = 2,
+    DST_BRANCH_CONVERT_AND_REDUCE = 3,
+    DST_BRANCH_GATHER = 4
+} dst_branch_t;
+typedef struct {
+    int32_t branch;       /* dst_branch_t: the line of the algorithm that applies */
+    int32_t out_kind;     /* dst_grad_kind_t of the output, -1 for an empty list */
+    int64_t out_rows;     /* rows of the output: vocab if dense, the concatenated row count if slices */
+    int64_t out_bytes;    /* bytes the output occupies (values, plus indices if slices) */
+    int32_t n_dense;      /* dense gradients in the list */
+    int32_t n_slices;     /* IndexedSlices gradients in the list */
+    int64_t n_slice_rows; /* their rows in total */
+    int32_t converts;     /* 1 when IndexedSlices are converted to dense (a workspace is needed) */
+    int32_t reserved;
+} dst_accum_plan_t;
+
+int dst_accumulate_plan(const dst_grad_t* grads, int32_t n, int64_t d, int64_t vocab, int32_t strategy,
+                        const dst_opts_t* opts, dst_accum_plan_t* plan);
+
+int dst_accumulate(const dst_grad_t* grads, int32_t n, int64_t d, int64_t vocab, int32_t strategy,
+                   void* out_dense, void* out_indices, void* out_values, int64_t out_capacity_rows,
+                   dst_stream_t stream, const dst_opts_t* opts, void* workspace, size_t workspace_bytes,
+                   dst_result_t* result, dst_accum_plan_t* plan);
+
+/*
  * Footprint report (Section 4: 11.4 GB gathered vs 139 MB dense at 64 processes).
  * n_rows_per_slice: HOST array of R row counts.  report: HOST.  Pure host arithmetic.
  */

@@ -7,9 +7,14 @@ operation runs in the library's CUDA kernels.  There is no CPU fallback: if
 the library has not been built, calls raise.
 """
 from .binding import (  # noqa: F401
+    DST_ACC_PROPOSED,
+    DST_ACC_SPARSE_AS_DENSE,
+    DST_ACC_STOCK,
     DST_STATUS,
     Densifier,
     DstError,
+    dst_accumulate,
+    dst_accumulate_plan,
     dst_bytes_report,
     dst_densify,
     dst_densify_concat,

@@ -1,6 +1,7 @@
 """ctypes marshalling for ``libdst_b200.so`` (see ``include/dst.h`` for the contract)."""
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 from typing import List, Optional, Sequence, Tuple
@@ -46,7 +47,21 @@ class _BytesReport(ctypes.Structure):
                 ("sparse_over_dense", ctypes.c_double), ("gather_all_over_dense", ctypes.c_double)]
 
 
+class _Grad(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("reserved", ctypes.c_int32), ("indices", ctypes.c_void_p),
+                ("values", ctypes.c_void_p), ("n_rows", ctypes.c_int64)]
+
+
+class _AccumPlan(ctypes.Structure):
+    _fields_ = [("branch", ctypes.c_int32), ("out_kind", ctypes.c_int32), ("out_rows", ctypes.c_int64),
+                ("out_bytes", ctypes.c_int64), ("n_dense", ctypes.c_int32), ("n_slices", ctypes.c_int32),
+                ("n_slice_rows", ctypes.c_int64), ("converts", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
 RESULT_BYTES = ctypes.sizeof(_Result)
+DST_GRAD_DENSE, DST_GRAD_SLICES = 0, 1
+DST_ACC_STOCK, DST_ACC_PROPOSED, DST_ACC_SPARSE_AS_DENSE = 0, 1, 2
+DST_BRANCH = {0: "empty", 1: "pass-through", 2: "reduce", 3: "convert+reduce", 4: "gather"}
 
 # name -> (restype, argtypes); also the list of symbols the header declares
 _vp, _i64, _i32, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
@@ -67,6 +82,10 @@ SYMBOLS = {
     "dst_kernel_launches": (ctypes.c_int64, []),
     "dst_bytes_report": (ctypes.c_int, [ctypes.POINTER(_i64), _i32, _i64, _i64, ctypes.POINTER(_Opts),
                                         ctypes.POINTER(_BytesReport)]),
+    "dst_accumulate_plan": (ctypes.c_int, [ctypes.POINTER(_Grad), _i32, _i64, _i64, _i32, ctypes.POINTER(_Opts),
+                                           ctypes.POINTER(_AccumPlan)]),
+    "dst_accumulate": (ctypes.c_int, [ctypes.POINTER(_Grad), _i32, _i64, _i64, _i32, _vp, _vp, _vp, _i64, _vp,
+                                      ctypes.POINTER(_Opts), _vp, _sz, _vp, ctypes.POINTER(_AccumPlan)]),
 }
 
 
@@ -287,6 +306,77 @@ def dst_densify_concat_host(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]],
                                          workspace.numel() * workspace.element_size(), _ptr(host_result))
     if rc != 0:
         raise DstError(rc, "dst_densify_concat_host")
+
+
+def _marshal_grads(grads, d: int, vocab: int, index_dtype, value_dtype, out_dtype):
+    """``grads``: a dense gradient is a [vocab, d] tensor, IndexedSlices are an (indices, values) pair."""
+    arr = (_Grad * max(len(grads), 1))()
+    for k, g in enumerate(grads):
+        if isinstance(g, torch.Tensor):
+            if g.numel() != vocab * d or not g.is_contiguous():
+                raise ValueError("a dense gradient must be contiguous [vocab, d]")
+            out_dtype = out_dtype or g.dtype
+            if g.dtype != out_dtype:
+                raise TypeError("all dense gradients must share one dtype")
+            arr[k].kind, arr[k].indices, arr[k].values, arr[k].n_rows = DST_GRAD_DENSE, None, g.data_ptr(), 0
+        else:
+            idx, val = g
+            index_dtype, value_dtype = index_dtype or idx.dtype, value_dtype or val.dtype
+            if idx.dtype != index_dtype or val.dtype != value_dtype:
+                raise TypeError("all IndexedSlices must share index and value dtypes")
+            _check_slice(idx, val, d, val.device)
+            arr[k].kind, arr[k].indices, arr[k].values, arr[k].n_rows = (DST_GRAD_SLICES, idx.data_ptr(),
+                                                                         val.data_ptr(), idx.shape[0])
+    return arr, index_dtype or torch.int64, value_dtype or out_dtype or torch.float32, out_dtype or value_dtype or torch.float32
+
+
+def _plan_dict(p: _AccumPlan) -> dict:
+    return {"branch": DST_BRANCH[p.branch], "out_kind": {0: "dense", 1: "slices", -1: None}[p.out_kind],
+            "out_rows": p.out_rows, "out_bytes": p.out_bytes, "n_dense": p.n_dense, "n_slices": p.n_slices,
+            "n_slice_rows": p.n_slice_rows, "converts": bool(p.converts)}
+
+
+def dst_accumulate_plan(grads, d: int, vocab: int, strategy: int = DST_ACC_PROPOSED, index_dtype=None,
+                        value_dtype=None, out_dtype=None) -> dict:
+    """``dst_accumulate_plan`` (include/dst.h): which branch of Algorithm 1 / Algorithm 2 / Listing 1 the list takes."""
+    lib = load_library()
+    arr, it, vt, ot = _marshal_grads(grads, d, vocab, index_dtype, value_dtype, out_dtype)
+    o = _opts(it, vt, ot)
+    p = _AccumPlan()
+    rc = lib.dst_accumulate_plan(arr, len(grads), d, vocab, strategy, ctypes.byref(o), ctypes.byref(p))
+    if rc != 0:
+        raise DstError(rc, "dst_accumulate_plan")
+    return _plan_dict(p)
+
+
+def dst_accumulate(grads, d: int, vocab: int, strategy: int = DST_ACC_PROPOSED, *,
+                   out_dense: Optional[torch.Tensor] = None, out_indices: Optional[torch.Tensor] = None,
+                   out_values: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                   result: Optional[torch.Tensor] = None, stream=None, index_dtype=None, value_dtype=None,
+                   out_dtype=None) -> dict:
+    """Enqueue ``dst_accumulate`` (include/dst.h).  Output buffers are the caller's; returns the plan."""
+    lib = load_library()
+    if out_dense is not None:
+        out_dtype = out_dtype or out_dense.dtype
+    arr, it, vt, ot = _marshal_grads(grads, d, vocab, index_dtype, value_dtype, out_dtype)
+    if out_dense is not None and (out_dense.dtype != ot or out_dense.numel() != vocab * d or not out_dense.is_contiguous()):
+        raise ValueError("out_dense must be contiguous [vocab, d] in the dense gradients' dtype")
+    cap = 0
+    if out_indices is not None and out_values is not None:
+        if out_indices.dtype != it or out_values.dtype != vt or not out_indices.is_contiguous() or not out_values.is_contiguous():
+            raise ValueError("out_indices / out_values must be contiguous and of the slices' dtypes")
+        cap = min(out_indices.shape[0], out_values.numel() // d if d else out_indices.shape[0])
+    o = _opts(it, vt, ot)
+    p = _AccumPlan()
+    dev = next((t.device for t in (out_dense, out_values, workspace) if t is not None), None)
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    with torch.cuda.device(dev) if dev is not None else contextlib.nullcontext():
+        rc = lib.dst_accumulate(arr, len(grads), d, vocab, strategy, _ptr(out_dense), _ptr(out_indices),
+                                _ptr(out_values), cap, _stream_handle(stream), ctypes.byref(o), _ptr(workspace),
+                                ws_bytes, _ptr(result), ctypes.byref(p))
+    if rc != 0:
+        raise DstError(rc, "dst_accumulate")
+    return _plan_dict(p)
 
 
 class Densifier:

@@ -10,7 +10,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(HERE, "libdst_b200.so")
-SOURCES = ["dst_api.cu", "dst_index_kernels.cu", "dst_front_cluster.cu", "dst_reduce_kernels.cu"]
+SOURCES = ["dst_api.cu", "dst_index_kernels.cu", "dst_front_cluster.cu", "dst_reduce_kernels.cu",
+           "dst_accumulate_kernels.cu"]
 HEADERS = [os.path.join(CSRC, "dst_common.cuh"), os.path.join(INCLUDE, "dst.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE]

@@ -2,6 +2,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <memory>
 #include <mutex>
 
 #include "dst_common.cuh"
@@ -320,6 +321,148 @@ int dst_densify_concat_host(const dst_slice_t* slices, int32_t R, int64_t d, int
         cudaMemcpyAsync(host_result, d_res, sizeof(dst_result_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
         return DST_ERR_CUDA;
     return DST_OK;
+}
+
+// ---- Algorithms 1 and 2, Listing 1: which branch a list of gradients takes ----
+int dst_accumulate_plan(const dst_grad_t* grads, int32_t n, int64_t d, int64_t vocab, int32_t strategy,
+                        const dst_opts_t* opts, dst_accum_plan_t* plan) {
+    if (!plan || n < 0 || d < 0 || vocab < 0 || (n > 0 && !grads)) return DST_ERR_INVALID_ARG;
+    if (!opts_ok(opts)) return opts ? DST_ERR_UNSUPPORTED : DST_ERR_INVALID_ARG;
+    if (strategy != DST_ACC_STOCK && strategy != DST_ACC_PROPOSED && strategy != DST_ACC_SPARSE_AS_DENSE)
+        return DST_ERR_INVALID_ARG;
+    dst_accum_plan_t p{};
+    for (int i = 0; i < n; ++i) {
+        if (grads[i].kind == DST_GRAD_DENSE) {
+            ++p.n_dense;
+        } else if (grads[i].kind == DST_GRAD_SLICES) {
+            if (grads[i].n_rows < 0) return DST_ERR_INVALID_ARG;
+            ++p.n_slices;
+            p.n_slice_rows += grads[i].n_rows;
+            if (p.n_slice_rows > kMaxRows) return DST_ERR_UNSUPPORTED;
+        } else {
+            return DST_ERR_INVALID_ARG;
+        }
+    }
+    const int64_t sv = (int64_t)dtype_size(opts->value_type), so = (int64_t)dtype_size(opts->out_type);
+    const int64_t si = (int64_t)index_size(opts->index_type);
+    // Listing 1 converts each IndexedSlices gradient before Algorithm 1 looks at the list
+    const bool all_dense = p.n_slices == 0 || strategy == DST_ACC_SPARSE_AS_DENSE;
+    bool dense_out;
+    if (n == 0) {
+        p.branch = DST_BRANCH_EMPTY;
+        p.out_kind = -1;
+        *plan = p;
+        return DST_OK;
+    } else if (n < 2) {
+        p.branch = DST_BRANCH_PASS_THROUGH;
+        dense_out = all_dense;
+    } else if (all_dense) {
+        p.branch = DST_BRANCH_REDUCE;
+        dense_out = true;
+    } else if (strategy == DST_ACC_PROPOSED && p.n_dense > 0) {
+        p.branch = DST_BRANCH_CONVERT_AND_REDUCE;
+        dense_out = true;
+    } else {
+        p.branch = DST_BRANCH_GATHER;
+        dense_out = false;
+    }
+    if (dense_out) {
+        p.out_kind = DST_GRAD_DENSE;
+        p.out_rows = vocab;
+        p.out_bytes = vocab * d * so;
+        p.converts = p.n_slices > 0;
+    } else {
+        p.out_kind = DST_GRAD_SLICES;
+        p.out_rows = p.n_slice_rows + (int64_t)p.n_dense * vocab;
+        p.out_bytes = p.out_rows * (d * sv + si);
+    }
+    *plan = p;
+    return DST_OK;
+}
+
+int dst_accumulate(const dst_grad_t* grads, int32_t n, int64_t d, int64_t vocab, int32_t strategy,
+                   void* out_dense, void* out_indices, void* out_values, int64_t out_capacity_rows,
+                   dst_stream_t stream, const dst_opts_t* opts, void* workspace, size_t workspace_bytes,
+                   dst_result_t* result, dst_accum_plan_t* plan_out) {
+    dst_accum_plan_t p{};
+    const int rc = dst_accumulate_plan(grads, n, d, vocab, strategy, opts, &p);
+    if (rc != DST_OK) return rc;
+    if (plan_out) *plan_out = p;
+    if (p.branch == DST_BRANCH_EMPTY || vocab == 0 || d == 0) return DST_OK;
+    for (int i = 0; i < n; ++i) {
+        if (!grads[i].values) { if (grads[i].kind == DST_GRAD_DENSE || grads[i].n_rows > 0) return DST_ERR_INVALID_ARG; }
+        if (grads[i].kind == DST_GRAD_SLICES && grads[i].n_rows > 0 && !grads[i].indices) return DST_ERR_INVALID_ARG;
+    }
+    const size_t sv = dtype_size(opts->value_type), so = dtype_size(opts->out_type), si = index_size(opts->index_type);
+
+    if (p.out_kind == DST_GRAD_SLICES) {
+        // gather (or the pass-through of one IndexedSlices gradient): concatenate in the order given
+        if (p.out_rows > out_capacity_rows || p.out_rows > kMaxRows) return DST_ERR_INVALID_ARG;
+        if (p.out_rows > 0 && (!out_indices || !out_values)) return DST_ERR_INVALID_ARG;
+        if (p.n_dense > 0 && opts->value_type != opts->out_type) return DST_ERR_UNSUPPORTED;
+        int64_t row = 0;
+        for (int i = 0; i < n; ++i) {
+            const bool dense = grads[i].kind == DST_GRAD_DENSE;
+            const int64_t rows = dense ? vocab : grads[i].n_rows;
+            if (rows == 0) continue;
+            char* oi = static_cast<char*>(out_indices) + size_t(row) * si;
+            char* ov = static_cast<char*>(out_values) + size_t(row) * size_t(d) * sv;
+            if (dense) {
+                // the rows of a dense tensor are its own indices (Section 3)
+                if (launch_iota(oi, rows, opts->index_type, sm_count(), stream) != cudaSuccess) return DST_ERR_CUDA;
+                ++g_launches;
+            } else if (cudaMemcpyAsync(oi, grads[i].indices, size_t(rows) * si, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
+                return DST_ERR_CUDA;
+            }
+            if (cudaMemcpyAsync(ov, grads[i].values, size_t(rows) * size_t(d) * sv, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+                return DST_ERR_CUDA;
+            row += rows;
+        }
+        return DST_OK;
+    }
+
+    // dense output: the dense gradients first, left to right, then the slices on top in one pass
+    if (!out_dense) return DST_ERR_INVALID_ARG;
+    const long long n_elems = (long long)vocab * d;
+    const void* partner = nullptr;          // what the slices are added to
+    if (p.n_dense == 1 && p.n_slices > 0) {
+        for (int i = 0; i < n; ++i) if (grads[i].kind == DST_GRAD_DENSE) partner = grads[i].values;
+    } else if (p.n_dense >= 1) {
+        SumParams sp{};
+        sp.out = out_dense; sp.n_elems = n_elems; sp.vector_ok = aligned16(out_dense);
+        bool first = true;
+        for (int i = 0; i < n; ++i) {
+            if (grads[i].kind != DST_GRAD_DENSE) continue;
+            sp.src[sp.k++] = grads[i].values;
+            sp.vector_ok = sp.vector_ok && aligned16(grads[i].values);
+            if (sp.k == kSumFanIn) {
+                if (launch_sum_dense(sp, opts->out_type, sm_count(), stream) != cudaSuccess) return DST_ERR_CUDA;
+                ++g_launches;
+                first = false;
+                sp.k = 0; sp.src[sp.k++] = out_dense; sp.vector_ok = aligned16(out_dense);   // carry on from the running sum
+            }
+        }
+        if (first ? sp.k >= 1 : sp.k >= 2) {
+            if (sp.k == 1 && sp.src[0] == out_dense) {
+                // a single dense gradient that already is the output
+            } else {
+                if (launch_sum_dense(sp, opts->out_type, sm_count(), stream) != cudaSuccess) return DST_ERR_CUDA;
+                ++g_launches;
+            }
+        }
+        partner = out_dense;
+    }
+    if (p.n_slices == 0) return DST_OK;
+    // convert_to_tensor of every IndexedSlices gradient (Listing 1), fused with the sum
+    dst_slice_t stack_slices[64];
+    dst_slice_t* sl = stack_slices;
+    std::unique_ptr<dst_slice_t[]> heap;
+    if (p.n_slices > 64) { heap.reset(new dst_slice_t[p.n_slices]); sl = heap.get(); }
+    int r = 0;
+    for (int i = 0; i < n; ++i)
+        if (grads[i].kind == DST_GRAD_SLICES) sl[r++] = dst_slice_t{grads[i].indices, grads[i].values, grads[i].n_rows};
+    return densify_impl(sl, p.n_slices, d, vocab, partner, out_dense, stream, opts, workspace, workspace_bytes,
+                        nullptr, nullptr, result);
 }
 
 int dst_bytes_report(const int64_t* n_rows_per_slice, int32_t R, int64_t d, int64_t vocab, const dst_opts_t* opts,

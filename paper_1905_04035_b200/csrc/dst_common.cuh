@@ -242,6 +242,17 @@ cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStrea
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
                           cudaStream_t stream);
 cudaError_t launch_scan(int index_type, const ScanParams& p, cudaStream_t stream);
+// ---- accumulation dispatcher (Algorithms 1 and 2) ----
+constexpr int kSumFanIn = 8;                // dense tensors summed per launch
+struct SumParams {
+    const void* src[kSumFanIn];
+    void* out;
+    long long n_elems;
+    int k;
+    int vector_ok;                          // every pointer 16-byte aligned
+};
+cudaError_t launch_sum_dense(const SumParams& p, int out_type, int sm_count, cudaStream_t stream);
+cudaError_t launch_iota(void* indices, long long n, int index_type, int sm_count, cudaStream_t stream);
 cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,
                                cudaStream_t stream);
 
