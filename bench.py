@@ -279,6 +279,58 @@ def time_device_warm(prob: DeviceProblem, steps: int, warmup: int):
     return t0.elapsed_time(t1) / steps
 
 
+def time_accumulate(device, steps: int, warmup: int, seed: int):
+    """The accumulation strategies of the paper on one rank's gradients of the tied weight (the big
+    configuration: the dense projection gradient and the two embedding lookups): Algorithm 1 gathers,
+    Algorithm 2 and Listing 1 convert and reduce; and the plain reduce branch on 2 and 8 dense tensors.
+    One library call per step, L2 flushed between steps, CUDA events around each call."""
+    import torch
+    import paper_1905_04035_b200 as dst
+    peak, _ = measured_peak()
+    w = make_workload("big", seed=seed)
+    tdt = {"f32": torch.float32, "i64": torch.int64}
+    dense = _dev_tensor(w.dense_in, w.out_dtype, device)
+    slices = [(_dev_tensor(i, w.index_dtype, device), _dev_tensor(v, w.value_dtype, device))
+              for i, v in zip(w.indices, w.values)]
+    n, d, vocab = w.n_rows_total, w.d, w.vocab
+    out_dense = torch.empty(vocab, d, device=device)
+    out_idx = torch.empty(vocab + n, dtype=torch.int64, device=device)
+    out_val = torch.empty(vocab + n, d, device=device)
+    ws = torch.empty(dst.dst_workspace_bytes(n, len(slices), d, vocab), dtype=torch.uint8, device=device)
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+    more = [torch.randn(vocab, d, device=device) * 0.02 for _ in range(7)]
+    dense_bytes, value_bytes, index_bytes = vocab * d * 4, n * d * 4, n * 8
+    cases = [
+        ("stock (Algorithm 1)", dst.DST_ACC_STOCK, [dense] + slices,
+         2 * (dense_bytes + value_bytes) + 2 * index_bytes + vocab * 8),       # copies: read + write; indices of the dense rows written
+        ("proposed (Algorithm 2)", dst.DST_ACC_PROPOSED, [dense] + slices, 2 * dense_bytes + value_bytes + index_bytes),
+        ("sparse_as_dense (Listing 1)", dst.DST_ACC_SPARSE_AS_DENSE, [dense] + slices, 2 * dense_bytes + value_bytes + index_bytes),
+        ("reduce, 2 dense", dst.DST_ACC_PROPOSED, [dense, more[0]], 3 * dense_bytes),
+        ("reduce, 8 dense", dst.DST_ACC_PROPOSED, [dense] + more, 9 * dense_bytes),
+    ]
+    rows = []
+    for name, strategy, grads, nbytes in cases:
+        def call():
+            return dst.dst_accumulate(grads, d, vocab, strategy, out_dense=out_dense, out_indices=out_idx,
+                                      out_values=out_val, workspace=ws)
+        for _ in range(warmup):
+            flush.zero_(); plan = call()
+        ev = []
+        l0 = dst.dst_kernel_launches()
+        for _ in range(steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); call(); b.record()
+            ev.append((a, b))
+        torch.cuda.synchronize()
+        ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+        rows.append({"strategy": name, "branch": plan["branch"], "out_kind": plan["out_kind"],
+                     "out_bytes": plan["out_bytes"], "ms_per_step": ms, "algorithmic_bytes": nbytes,
+                     "gbs": nbytes / ms / 1e6, "frac_of_hbm_peak": nbytes / ms / 1e6 / peak,
+                     "gpu_launches_per_step": (dst.dst_kernel_launches() - l0) / steps})
+    return rows
+
+
 def time_e2e(w, device, steps: int, warmup: int):
     """Same metric through the host entry point: pinned host buffers, H2D and D2H inside the timed region."""
     import torch
@@ -483,6 +535,10 @@ def main():
                                              "algorithmic_bytes", "reduce_kernel_ms", "reduce_kernel_frac", "l2", "eager_ms_per_step", "warm_ms_per_step",
                                              "n_unique", "max_segment", "status")})
 
+    accumulate = None
+    if rank == 0 and world == 1 and not args.headline_only:
+        accumulate = time_accumulate(device, min(args.steps, 50), args.warmup, args.seed)
+
     cpu = cpu_threads = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         info = time_oracle(w, max_rows=None if w.n_rows_total <= 700000 else 700000)
@@ -514,7 +570,7 @@ def main():
                          "kernel": "k_reduce_rows", "of": head["peak_source"],
                          "kernel_ms": head["reduce_kernel_ms"]},
             "e2e": e2e, "gpu_launches": head["launches"], "clocks": head["clocks"],
-            "cpu_baseline": cpu, "cpu_baseline_threads": cpu_threads, "bytes_report": rep, "all_configs": others,
+            "cpu_baseline": cpu, "cpu_baseline_threads": cpu_threads, "bytes_report": rep, "all_configs": others, "accumulate": accumulate,
             "parity": {"status": head["status"], "n_unique": head["n_unique"], "max_segment": head["max_segment"]},
         }
         print(json.dumps(line))
