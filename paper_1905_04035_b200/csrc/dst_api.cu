@@ -3,6 +3,7 @@
 
 #include <atomic>
 #include <memory>
+#include <new>
 #include <mutex>
 
 #include "dst_common.cuh"
@@ -457,7 +458,11 @@ int dst_accumulate(const dst_grad_t* grads, int32_t n, int64_t d, int64_t vocab,
     dst_slice_t stack_slices[64];
     dst_slice_t* sl = stack_slices;
     std::unique_ptr<dst_slice_t[]> heap;
-    if (p.n_slices > 64) { heap.reset(new dst_slice_t[p.n_slices]); sl = heap.get(); }
+    if (p.n_slices > 64) {
+        heap.reset(new (std::nothrow) dst_slice_t[p.n_slices]);
+        if (!heap) return DST_ERR_INVALID_ARG;
+        sl = heap.get();
+    }
     int r = 0;
     for (int i = 0; i < n; ++i)
         if (grads[i].kind == DST_GRAD_SLICES) sl[r++] = dst_slice_t{grads[i].indices, grads[i].values, grads[i].n_rows};
