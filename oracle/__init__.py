@@ -1,6 +1,8 @@
 """CPU oracle (test infrastructure only; never imported by the product path)."""
 from .dst_oracle import (  # noqa: F401
     OracleResult,
+    SgdResult,
+    apply_sgd,
     build_oracle_library,
     bytes_report,
     densify,

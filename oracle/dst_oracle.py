@@ -121,6 +121,29 @@ def densify(indices: Sequence[np.ndarray], values: Sequence[np.ndarray], d: int,
                         int(n_bad.value), int(cnt.max()) if vocab else 0)
 
 
+@dataclasses.dataclass
+class SgdResult:
+    weight: np.ndarray       # [vocab, d] float64: the updated weight, unrounded
+    mag: np.ndarray          # [vocab, d] float64: |w| + lr * sum of |gradient terms| (tolerance scale)
+    out: np.ndarray          # [vocab, d] float32: rounded once
+    grad: OracleResult       # the dense gradient that was applied
+
+
+def apply_sgd(indices: Sequence[np.ndarray], values: Sequence[np.ndarray], d: int, vocab: int,
+              dense_in: Optional[np.ndarray], weight: np.ndarray, lr: float) -> SgdResult:
+    """The step that follows accumulation in the paper's training loop (Section 4: the optimizer the
+    distributed wrapper hands the accumulated gradients to), for plain SGD on the tied weight:
+
+        weight[v, c] <- weight[v, c] - lr * (dense_in[v, c] + sum of the value rows naming v)
+
+    Written as exactly that: the pinned scatter-sum of ``densify`` in fp64, then one fp64 multiply-subtract
+    per element.  fp32 tensors only."""
+    g = densify(indices, values, d, vocab, dense_in)
+    w = np.asarray(weight, np.float32).reshape(vocab, d).astype(np.float64)
+    new = w - float(lr) * g.acc
+    return SgdResult(new, np.abs(w) + abs(float(lr)) * g.mag, new.astype(np.float32), g)
+
+
 def round_bf16(x: float) -> int:
     return int(_load().dst_oracle_round_bf16(float(x)))
 
