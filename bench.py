@@ -328,6 +328,34 @@ def time_accumulate(device, steps: int, warmup: int, seed: int):
                      "out_bytes": plan["out_bytes"], "ms_per_step": ms, "algorithmic_bytes": nbytes,
                      "gbs": nbytes / ms / 1e6, "frac_of_hbm_peak": nbytes / ms / 1e6 / peak,
                      "gpu_launches_per_step": (dst.dst_kernel_launches() - l0) / steps})
+    # the SGD step fused into the same pass, against densify followed by a separate update of the weight
+    weight = torch.randn(vocab, d, device=device)
+    lr = 0.1
+
+    def fused():
+        dst.dst_densify_apply_sgd(slices, d, vocab, dense, weight, lr, ws)
+
+    def separate():
+        dst.dst_densify_concat(slices, d, vocab, dense, out_dense, ws)
+        weight.add_(out_dense, alpha=-lr)
+
+    for name, fn, nbytes in (("densify + SGD step, fused (dst_densify_apply_sgd)", fused, 3 * dense_bytes + value_bytes + index_bytes),
+                             ("densify, then a separate weight update", separate, 5 * dense_bytes + value_bytes + index_bytes)):
+        for _ in range(warmup):
+            flush.zero_(); fn()
+        ev = []
+        l0 = dst.dst_kernel_launches()
+        for _ in range(steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            ev.append((a, b))
+        torch.cuda.synchronize()
+        ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+        rows.append({"strategy": name, "branch": "convert+reduce+apply", "out_kind": "weight", "out_bytes": dense_bytes,
+                     "ms_per_step": ms, "algorithmic_bytes": nbytes, "gbs": nbytes / ms / 1e6,
+                     "frac_of_hbm_peak": nbytes / ms / 1e6 / peak,
+                     "gpu_launches_per_step": (dst.dst_kernel_launches() - l0) / steps})
     return rows
 
 

@@ -131,6 +131,24 @@ int dst_densify_concat(const dst_slice_t* slices, int32_t R, int64_t d, int64_t 
                        void* unique_rows, int32_t* counts, dst_result_t* result);
 
 /*
+ * dst_densify_concat fused with the step that follows accumulation in the training loop (Section 4:
+ * the optimizer the accumulated gradient is handed to), for plain SGD on the tied weight:
+ *
+ *     weight[v, c] <- weight[v, c] - lr * (dense_in[v, c] + sum of the value rows that name v)
+ *
+ * The dense gradient is never written: every weight row is read once and written once, next to the
+ * one read of dense_in and of the value rows.  fp32 only (value_type and out_type DST_F32, otherwise
+ * DST_ERR_UNSUPPORTED); `weight` is [vocab, d], updated in place, and must not be dense_in.  The
+ * gradient of a row is summed in the order dst_densify_concat uses, dense_in last, then one fused
+ * multiply-add takes the step.  All other arguments, the optional outputs and the error behaviour are
+ * those of dst_densify_concat; rows with an out-of-range index are skipped and reported.
+ */
+int dst_densify_apply_sgd(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab,
+                          const void* dense_in, void* weight, float lr, dst_stream_t stream,
+                          const dst_opts_t* opts, void* workspace, size_t workspace_bytes,
+                          void* unique_rows, int32_t* counts, dst_result_t* result);
+
+/*
  * dst_densify without a caller-supplied workspace.  (The paper has no counterpart:
  * this entry point exists for the sake of callers, not of the method.)
  *

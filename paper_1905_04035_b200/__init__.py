@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     dst_accumulate_plan,
     dst_bytes_report,
     dst_densify,
+    dst_densify_apply_sgd,
     dst_densify_concat,
     dst_densify_concat_host,
     dst_densify_static,

@@ -73,6 +73,8 @@ SYMBOLS = {
                                    _vp, _vp, _vp]),
     "dst_densify_concat": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, _vp,
                                           ctypes.POINTER(_Opts), _vp, _sz, _vp, _vp, _vp]),
+    "dst_densify_apply_sgd": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, ctypes.c_float, _vp,
+                                             ctypes.POINTER(_Opts), _vp, _sz, _vp, _vp, _vp]),
     "dst_densify_static": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i64, _vp, _vp, _vp, ctypes.POINTER(_Opts),
                                           _vp, _vp, _vp]),
     "dst_host_staging_bytes": (_sz, [_i64, _i64, _i64, ctypes.POINTER(_Opts)]),
@@ -228,6 +230,35 @@ def dst_densify_concat(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]], d: i
                                     _ptr(unique_rows), _ptr(counts), _ptr(result))
     if rc != 0:
         raise DstError(rc, "dst_densify_concat")
+
+
+def dst_densify_apply_sgd(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]], d: int, vocab: int,
+                          dense_in: Optional[torch.Tensor], weight: torch.Tensor, lr: float, workspace: torch.Tensor,
+                          unique_rows: Optional[torch.Tensor] = None, counts: Optional[torch.Tensor] = None,
+                          result: Optional[torch.Tensor] = None, stream=None,
+                          index_dtype: Optional[torch.dtype] = None) -> None:
+    """Enqueue ``dst_densify_apply_sgd`` (include/dst.h): weight -= lr * (dense_in + densified slices), fp32."""
+    lib = load_library()
+    R = len(slices)
+    index_dtype = slices[0][0].dtype if R else (index_dtype or torch.int64)
+    arr = (_Slice * max(R, 1))()
+    for r, (idx, val) in enumerate(slices):
+        if idx.dtype != index_dtype or val.dtype != torch.float32:
+            raise TypeError("all slices must share the index dtype and hold float32 values")
+        _check_slice(idx, val, d, weight.device)
+        arr[r].indices, arr[r].values, arr[r].n_rows = idx.data_ptr(), val.data_ptr(), idx.shape[0]
+    if weight.dtype != torch.float32 or weight.numel() != vocab * d or not weight.is_contiguous():
+        raise ValueError("weight must be contiguous float32 [vocab, d]")
+    if dense_in is not None and (dense_in.dtype != torch.float32 or dense_in.numel() != vocab * d
+                                 or not dense_in.is_contiguous()):
+        raise ValueError("dense_in must be contiguous float32 [vocab, d]")
+    o = _opts(index_dtype, torch.float32, torch.float32)
+    with torch.cuda.device(weight.device):
+        rc = lib.dst_densify_apply_sgd(arr, R, d, vocab, _ptr(dense_in), _ptr(weight), float(lr), _stream_handle(stream),
+                                       ctypes.byref(o), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                       _ptr(unique_rows), _ptr(counts), _ptr(result))
+    if rc != 0:
+        raise DstError(rc, "dst_densify_apply_sgd")
 
 
 def dst_densify(indices: torch.Tensor, values: torch.Tensor, d: int, vocab: int,

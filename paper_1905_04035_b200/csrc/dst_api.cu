@@ -39,8 +39,11 @@ static int sm_count() {
 
 static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
                         void* out, cudaStream_t stream, const dst_opts_t* opts, void* workspace,
-                        size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
+                        size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result,
+                        bool apply = false, float lr = 0.f) {
     if (!opts_ok(opts)) return opts ? DST_ERR_UNSUPPORTED : DST_ERR_INVALID_ARG;
+    if (apply && (opts->value_type != DST_F32 || opts->out_type != DST_F32)) return DST_ERR_UNSUPPORTED;
+    if (apply && out && out == dense_in) return DST_ERR_INVALID_ARG;   // the weight is not its own gradient
     if (R < 0 || d < 0 || vocab < 0 || (R > 0 && !slices)) return DST_ERR_INVALID_ARG;
     if (vocab > kMaxVocab) return DST_ERR_UNSUPPORTED;
     int64_t n_total = 0;
@@ -106,6 +109,8 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         fp.copy_src = dense_in; fp.copy_dst = out;
         fp.copy_bytes = int64_t(vocab) * d * int64_t(dtype_size(opts->out_type));
         fp.copy_clusters = compact && out != dense_in ? (sm_count() - kClusterCtas) / kClusterCtas : 0;
+        fp.copy_apply = apply ? 1 : 0; fp.copy_lr = lr;
+        if (apply && !dense_in) fp.copy_clusters = 0;   // nothing to take from the rows nobody names
         if (launch_front_cluster(opts->index_type, fp, stream) != cudaSuccess) return DST_ERR_CUDA;
         ++g_launches;
         perm = pos[0];
@@ -159,6 +164,7 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     a.chunk_max = int(L.chunk_max); a.upper_max = int(L.upper_max);
     a.W = a.ncb = a.slot_bytes = a.n_slots = 0;   // set by the launcher
     a.compact = compact ? 1 : 0;
+    a.apply = apply ? 1 : 0; a.lr = lr;
     a.urow = reinterpret_cast<const int*>(ws + L.off_urow);
     a.uoff = reinterpret_cast<const int*>(ws + L.off_uoff);
     if (t_ev_before && cudaEventRecord(t_ev_before, stream) != cudaSuccess) return DST_ERR_CUDA;
@@ -245,6 +251,13 @@ int dst_densify_concat(const dst_slice_t* slices, int32_t R, int64_t d, int64_t 
                        size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
     return densify_impl(slices, R, d, vocab, dense_in, out, stream, opts, workspace, workspace_bytes, unique_rows,
                         counts, result);
+}
+
+int dst_densify_apply_sgd(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
+                          void* weight, float lr, dst_stream_t stream, const dst_opts_t* opts, void* workspace,
+                          size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
+    return densify_impl(slices, R, d, vocab, dense_in, weight, stream, opts, workspace, workspace_bytes, unique_rows,
+                        counts, result, true, lr);
 }
 
 int dst_densify_static(const void* indices, const void* values, int64_t n_rows, int64_t d, int64_t vocab,

@@ -128,6 +128,8 @@ struct MainArgs {
     int ncb;         // column blocks per row
     int slot_bytes;
     int n_slots;
+    int apply;       // 1: `out` holds a weight and gets the SGD step (fp32 only), see dst_densify_apply_sgd
+    float lr;        // learning rate of that step
     int compact;     // out already holds dense_in (or zeros) everywhere: the row batches list only the named rows
 };
 
@@ -237,6 +239,8 @@ struct FrontParams {
     void* copy_dst;            // out
     long long copy_bytes;      // vocab * d * sizeof(out element), a multiple of 16
     int copy_clusters;         // extra clusters that fill out while the first one does the index work
+    int copy_apply;            // 1: the extra clusters take the dense part of the SGD step, out -= copy_lr * dense_in (fp32)
+    float copy_lr;
 };
 cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStream_t stream);
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,

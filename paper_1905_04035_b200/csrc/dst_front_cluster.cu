@@ -49,6 +49,8 @@ struct FrontArgs {
     const uint4* copy_src;     // clusters after the first: out = dense_in (or zeros), 16 bytes per thread and step
     uint4* copy_dst;
     long long copy_vecs;
+    int copy_apply;            // out -= copy_lr * dense_in instead of out = dense_in (fp32 tensors)
+    float copy_lr;
 };
 
 constexpr int kFrontWarps = kFrontThreads / 32;
@@ -130,7 +132,25 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
         // and this copy, most of the bytes of the whole operation, hides the index work entirely.
         const long long stride = (long long)(gridDim.x - kClusterCtas) * kFrontThreads;
         long long i = (long long)(blockIdx.x - kClusterCtas) * kFrontThreads + threadIdx.x;
-        if (f.copy_src) {
+        if (f.copy_src && f.copy_apply) {
+            // the dense part of the SGD step for every row: weight -= lr * dense gradient
+            const float4* src = reinterpret_cast<const float4*>(f.copy_src);
+            float4* dst = reinterpret_cast<float4*>(f.copy_dst);
+            const float nlr = -f.copy_lr;
+            for (; i + 3 * stride < f.copy_vecs; i += 4 * stride) {
+                float4 g[4], w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) { g[q] = __ldcs(src + i + q * stride); w[q] = __ldcs(dst + i + q * stride); }
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    __stcs(dst + i + q * stride, make_float4(fmaf(nlr, g[q].x, w[q].x), fmaf(nlr, g[q].y, w[q].y),
+                                                            fmaf(nlr, g[q].z, w[q].z), fmaf(nlr, g[q].w, w[q].w)));
+            }
+            for (; i < f.copy_vecs; i += stride) {
+                const float4 g = __ldcs(src + i), w = __ldcs(dst + i);
+                __stcs(dst + i, make_float4(fmaf(nlr, g.x, w.x), fmaf(nlr, g.y, w.y), fmaf(nlr, g.z, w.z), fmaf(nlr, g.w, w.w)));
+            }
+        } else if (f.copy_src) {
             for (; i + 7 * stride < f.copy_vecs; i += 8 * stride) {
                 uint4 v[8];
 #pragma unroll
@@ -404,6 +424,7 @@ cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStrea
     f.batch_units = p.batch_units; f.batch_max = p.batch_max; f.nodecnt_words = p.nodecnt_words;
     f.copy_src = static_cast<const uint4*>(p.copy_src); f.copy_dst = static_cast<uint4*>(p.copy_dst);
     f.copy_vecs = p.copy_bytes / 16;
+    f.copy_apply = p.copy_apply; f.copy_lr = p.copy_lr;
     const int per_warp = (p.n_total + kClusterCtas * kFrontWarps - 1) / (kClusterCtas * kFrontWarps);
     f.lw = (per_warp + 31) / 32 * 32;
     if (f.lw < 32) f.lw = 32;

@@ -174,7 +174,9 @@ struct UnitBlock {
     int y;               // output row (kUnitFinal) or chunk id (kUnitChunkEnd)
 };
 
-template <typename VT, typename OT, int K>
+// APPLY: instead of writing the accumulated gradient, take the SGD step on the weight that `out` holds
+// (fp32 rows only): out <- out - lr * (dense_in + sum of value rows).
+template <typename VT, typename OT, int K, bool APPLY = false>
 struct WarpPipe {
     static constexpr int VC = 16 / sizeof(VT);     // columns per 16-byte group of a value row
     const MainArgs& a;
@@ -367,13 +369,15 @@ struct WarpPipe {
             constexpr bool kDenseInRing = sizeof(VT) == 4 && sizeof(OT) == 4;
             const float* dense_row = nullptr;
             if constexpr (kDenseInRing)
-                if (root && a.dense_in) dense_row = static_cast<const float*>(a.dense_in) + (long long)hi.row * a.d + cb;
+                if (root && a.dense_in && !(APPLY && a.compact))   // a pre-filled weight already holds the dense part of the step
+                    dense_row = static_cast<const float*>(a.dense_in) + (long long)hi.row * a.d + cb;
             if (!sum_children(acc, child_first + parent * kFanIn, n_children, cb, wcols, dense_row)) return false;
             if (root) {
                 // The output may be the dense input itself, so the compiler keeps loads and stores in
                 // program order: read the whole dense row first, then store, or every column group
                 // pays its own trip to memory.
-                const OT* din = kDenseInRing ? nullptr : static_cast<const OT*>(a.dense_in);
+                const OT* din = APPLY ? static_cast<const OT*>(a.out)            // the weight row
+                                      : (kDenseInRing ? nullptr : static_cast<const OT*>(a.dense_in));
                 OT* out = static_cast<OT*>(a.out) + (long long)hi.row * a.d + cb;
                 constexpr int KH = (sizeof(VT) == 2 && K >= 4) ? K / 2 : K;
 #pragma unroll
@@ -388,7 +392,12 @@ struct WarpPipe {
 #pragma unroll
                     for (int k = 0; k < KH; ++k) {
                         const int c = col(h0 + k);
-                        add(acc[h0 + k], dn[k]);
+                        if constexpr (APPLY) {
+#pragma unroll
+                            for (int i = 0; i < VC; ++i) acc[h0 + k].x[i] = fmaf(-a.lr, acc[h0 + k].x[i], dn[k].x[i]);
+                        } else {
+                            add(acc[h0 + k], dn[k]);
+                        }
                         if (c < wcols) store_out(out + c, acc[h0 + k]);
                     }
                 }
@@ -445,12 +454,18 @@ struct WarpPipe {
                 for (int k = 0; k < K; ++k) {
                     const int c = col(k);
                     zero(dn[k]);
-                    if (a.dense_in && c < wcols) load_elems(reinterpret_cast<const OT*>(sp) + c, dn[k]);
+                    if ((APPLY || a.dense_in) && c < wcols) load_elems(reinterpret_cast<const OT*>(sp) + c, dn[k]);
                 }
 #pragma unroll
                 for (int k = 0; k < K; ++k) {
                     const int c = col(k);
-                    if (!(kind & kUnitCopy)) add(dn[k], acc[k]);
+                    if constexpr (APPLY) {
+                        // the slot holds the weight row; acc holds the whole gradient of the row
+#pragma unroll
+                        for (int i = 0; i < VC; ++i) dn[k].x[i] = fmaf(-a.lr, acc[k].x[i], dn[k].x[i]);
+                    } else {
+                        if (!(kind & kUnitCopy)) add(dn[k], acc[k]);
+                    }
                     if (c < wcols) store_out(orow + c, dn[k]);
                     zero(acc[k]);
                 }
@@ -504,7 +519,9 @@ struct WarpPipe {
         }
         const int o_next = __shfl_down_sync(0xFFFFFFFFu, o, 1);
         const int cnt = lane < nrows ? o_next - o : 0;
-        const int nunits = (lane < nrows && cnt <= a.chunk) ? cnt + 1 : 0;   // heavy rows belong to the chunk items
+        // APPLY, output not pre-filled: the dense row is one more unit to add, before the weight row closes the row
+        const bool dense_unit = APPLY && a.dense_in && !a.compact;
+        const int nunits = (lane < nrows && cnt <= a.chunk) ? cnt + 1 + (dense_unit ? 1 : 0) : 0;   // heavy rows belong to the chunk items
         int incl = nunits;
 #pragma unroll
         for (int s = 1; s < 32; s <<= 1) {
@@ -535,9 +552,16 @@ struct WarpPipe {
                         b.bytes = (unsigned)(wcols * (long long)sizeof(VT));
                         b.kind = kUnitAdd;
                     }
+                } else if (dense_unit && e == ci) {
+                    b.src = static_cast<const OT*>(a.dense_in) + (long long)b.y * a.d + cb;
+                    b.bytes = (unsigned)(wcols * (long long)sizeof(OT));
+                    b.kind = kUnitAdd;
                 } else {
                     b.kind = kUnitFinal | (ci == 0 ? kUnitCopy : 0);
-                    if (a.dense_in) {
+                    if constexpr (APPLY) {
+                        b.src = static_cast<const OT*>(a.out) + (long long)b.y * a.d + cb;
+                        b.bytes = (unsigned)(wcols * (long long)sizeof(OT));
+                    } else if (a.dense_in) {
                         b.src = static_cast<const OT*>(a.dense_in) + (long long)b.y * a.d + cb;
                         b.bytes = (unsigned)(wcols * (long long)sizeof(OT));
                     }
@@ -588,7 +612,7 @@ struct WarpPipe {
     }
 };
 
-template <typename VT, typename OT, int K>
+template <typename VT, typename OT, int K, bool APPLY = false>
 __global__ void __launch_bounds__(kPipeThreads, sizeof(VT) == 2 ? 4 : 2)
 k_reduce_rows(const __grid_constant__ MainArgs a) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -619,7 +643,7 @@ k_reduce_rows(const __grid_constant__ MainArgs a) {
     __syncthreads();
     {
         char* my_ring = slot_base + (size_t)warp * (size_t)a.n_slots * (size_t)a.slot_bytes;
-        WarpPipe<VT, OT, K> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort, tabs);
+        WarpPipe<VT, OT, K, APPLY> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort, tabs);
         // after a failed wait in an earlier kernel the tables are not to be trusted: touch nothing
         if (*reinterpret_cast<volatile int*>(&a.hdr->status) != DST_ERR_TIMEOUT) pipe.run();
     }
@@ -646,14 +670,14 @@ k_reduce_rows_scalar(const MainArgs a) {
         const int v = (int)(e / a.d);
         const long long c = e - (long long)v * a.d;
         const int beg = a.offsets[v], end = a.offsets[v + 1];
-        if (beg == end) { out[e] = din ? din[e] : OT(0.f); continue; }
+        if (beg == end && !a.apply) { out[e] = din ? din[e] : OT(0.f); continue; }
         float acc = 0.f;
         for (int j = beg; j < end; ++j) {
             unsigned p = a.perm[j];
             if (p < (unsigned)a.n_total) acc += (float)resolve_row<VT>(a, p)[c];
         }
         if (din) acc += (float)din[e];
-        out[e] = OT(acc);
+        out[e] = a.apply ? OT(fmaf(-a.lr, acc, (float)out[e])) : OT(acc);
     }
 }
 
@@ -662,23 +686,23 @@ k_reduce_rows_scalar(const MainArgs a) {
 // index lookup, a node of a combine tree), which is what a short call is made of.
 constexpr long long kInFlightBytes = 14ll << 20;
 
-template <typename VT, typename OT, int K>
+template <typename VT, typename OT, int K, bool APPLY>
 static cudaError_t launch_pipe(MainArgs a, int sm_count, cudaStream_t stream) {
     auto smem_for = [&](int slots) { return size_t(kPipeHeaderReserve) + size_t(kPipeWarps) * size_t(slots) * size_t(a.slot_bytes); };
-    cudaError_t e = cudaFuncSetAttribute(k_reduce_rows<VT, OT, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_for(kPipeSlots));
+    cudaError_t e = cudaFuncSetAttribute(k_reduce_rows<VT, OT, K, APPLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_for(kPipeSlots));
     if (e != cudaSuccess) return e;
     int resident = 0;                                    // CTAs of this variant an SM holds with full rings
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, k_reduce_rows<VT, OT, K>, kPipeThreads, smem_for(kPipeSlots));
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, k_reduce_rows<VT, OT, K, APPLY>, kPipeThreads, smem_for(kPipeSlots));
     if (e != cudaSuccess) return e;
     if (resident < 1) return cudaErrorLaunchOutOfResources;
     const int grid = sm_count * resident;
     const long long per_slot = (long long)grid * kPipeWarps * a.slot_bytes;
     long long slots = kInFlightBytes / per_slot;
     a.n_slots = (int)(slots < 2 ? 2 : (slots > kPipeSlots ? kPipeSlots : slots));
-    return launch_pdl(k_reduce_rows<VT, OT, K>, dim3(grid), dim3(kPipeThreads), smem_for(a.n_slots), stream, a);
+    return launch_pdl(k_reduce_rows<VT, OT, K, APPLY>, dim3(grid), dim3(kPipeThreads), smem_for(a.n_slots), stream, a);
 }
 
-template <typename VT, typename OT>
+template <typename VT, typename OT, bool APPLY = false>
 static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaStream_t stream) {
     if (!vector_ok) {
         long long total = (long long)a.vocab * a.d;
@@ -691,14 +715,18 @@ static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaSt
     const PipeShape ps = pipe_shape((int)sizeof(VT), (int)sizeof(OT), a.d);
     a.W = ps.W; a.ncb = ps.ncb; a.slot_bytes = ps.slot_bytes; a.n_slots = ps.n_slots;
     constexpr int kMaxK = sizeof(VT) == 4 ? 8 : 4;
-    if (ps.K == 1) return launch_pipe<VT, OT, 1>(a, sm_count, stream);
-    if (ps.K == 2) return launch_pipe<VT, OT, 2>(a, sm_count, stream);
-    if (ps.K == 4 || kMaxK == 4) return launch_pipe<VT, OT, 4>(a, sm_count, stream);
-    return launch_pipe<VT, OT, kMaxK>(a, sm_count, stream);
+    if (ps.K == 1) return launch_pipe<VT, OT, 1, APPLY>(a, sm_count, stream);
+    if (ps.K == 2) return launch_pipe<VT, OT, 2, APPLY>(a, sm_count, stream);
+    if (ps.K == 4 || kMaxK == 4) return launch_pipe<VT, OT, 4, APPLY>(a, sm_count, stream);
+    return launch_pipe<VT, OT, kMaxK, APPLY>(a, sm_count, stream);
 }
 
 cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,
                                cudaStream_t stream) {
+    if (a.apply) {
+        if (value_type != DST_F32 || out_type != DST_F32) return cudaErrorInvalidValue;
+        return launch_typed<float, float, true>(a, vector_ok, sm_count, stream);
+    }
     if (value_type == DST_F32 && out_type == DST_F32) return launch_typed<float, float>(a, vector_ok, sm_count, stream);
     if (value_type == DST_F32 && out_type == DST_BF16) return launch_typed<float, __nv_bfloat16>(a, vector_ok, sm_count, stream);
     if (value_type == DST_BF16 && out_type == DST_F32) return launch_typed<__nv_bfloat16, float>(a, vector_ok, sm_count, stream);
