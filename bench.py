@@ -509,6 +509,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager calls instead of CUDA-graph replays")
+    ap.add_argument("--accumulate-only", action="store_true",
+                    help="only the accumulation-strategy and fused-SGD calls (prints their rows, one GPU)")
     ap.add_argument("--scale", type=float, default=1.0,
                     help="shrink the rows per slice (profiling captures on a small case); 1.0 = the named configuration")
     ap.add_argument("--reference-rows", type=int, default=163840,
@@ -536,6 +538,11 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
         dist_ctx = dist
+
+    if args.accumulate_only:
+        if rank == 0:
+            print(json.dumps({"accumulate": time_accumulate(device, min(args.steps, 50), args.warmup, args.seed)}))
+        return
 
     # every rank is an independent replica with its own seed (the path has no exchange step)
     from paper_1905_04035_b200.replicas import combine_over_ranks, replica_seed
