@@ -170,3 +170,24 @@ def test_accumulate_in_place_and_capacity_check():
     small_v = torch.empty(10, d, device=dev)
     with pytest.raises(dst.DstError):
         dst.dst_accumulate([dense, sl], d, vocab, dst.DST_ACC_STOCK, out_indices=small_i, out_values=small_v)
+
+
+@pytest.mark.gpu
+def test_accumulate_paper_case_at_full_size():
+    """One rank's gradients of the tied weight at the size the benchmark times (vocab 33708, d 1024, two lookups of
+    12,800 rows): the proposed strategy is one fused densify; the stock strategy gathers vocab + 25,600 rows."""
+    from paper_1905_04035_b200.workloads import make_workload
+    w = make_workload("big")
+    grads = [ao.Grad(w.dense_in)] + [ao.Grad(v, i) for i, v in zip(w.indices, w.values)]
+    ref = ao.accumulate(grads, w.d, w.vocab, ao.PROPOSED)
+    plan, out_dense, _, _, result, launches = run_gpu(grads, w.d, w.vocab, dst.DST_ACC_PROPOSED)
+    assert plan["branch"] == "convert+reduce" and launches == 2          # index cluster + row reduction, no sum kernel
+    mag = np.abs(w.dense_in).astype(np.float64)
+    for i, v in zip(w.indices, w.values):
+        np.add.at(mag, i, np.abs(v.astype(np.float64)))
+    assert np.all(np.abs(widen(out_dense) - ref.grad.values) <= 1e-5 * mag + 1e-7)
+    plan, _, out_idx, out_val, _, _ = run_gpu(grads, w.d, w.vocab, dst.DST_ACC_STOCK)
+    assert plan["branch"] == "gather" and plan["out_rows"] == w.vocab + w.n_rows_total
+    assert plan["out_bytes"] == (w.vocab + w.n_rows_total) * (w.d * 4 + 8)
+    st = ao.accumulate(grads, w.d, w.vocab, ao.STOCK).grad
+    assert np.array_equal(out_idx.cpu().numpy(), st.indices) and np.array_equal(out_val.cpu().numpy(), st.values)

@@ -45,7 +45,7 @@ def check(indices, values, d, vocab, dense, weight, lr, exact=False):
     return got, ref, result
 
 
-@pytest.mark.parametrize("name", ["tiny", "base"])
+@pytest.mark.parametrize("name", ["tiny", "base", "big"])
 def test_paper_configurations(name):
     w = make_workload(name)                                         # one-cluster index path, output pre-filled
     weight = np.random.default_rng(1).normal(0, 1, size=(w.vocab, w.d)).astype(np.float32)
