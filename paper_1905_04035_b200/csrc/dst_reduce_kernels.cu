@@ -199,15 +199,13 @@ struct WarpPipe {
 
     __device__ __forceinline__ int col(int k) const { return (k * 32 + lane) * VC; }
 
-    // unit j of the block goes into the next slot (lane 0 talks to the copy engine)
+    // unit j of the block goes into the next slot
     __device__ __forceinline__ void issue(const UnitBlock& b, int j) {
-        const unsigned long long s = __shfl_sync(0xFFFFFFFFu, reinterpret_cast<unsigned long long>(b.src), j);
-        const unsigned bytes = __shfl_sync(0xFFFFFFFFu, b.bytes, j);
-        if (lane == 0) {
+        if (lane == j) {                                  // the lane that holds the unit talks to the copy engine
             const unsigned bar = bars + 8u * (unsigned)islot;
-            if (bytes) {
-                mbar_arrive_expect_tx(bar, bytes);
-                bulk_load(ring + (unsigned)islot * (unsigned)a.slot_bytes, reinterpret_cast<const void*>(s), bytes, bar);
+            if (b.bytes) {
+                mbar_arrive_expect_tx(bar, b.bytes);
+                bulk_load(ring + (unsigned)islot * (unsigned)a.slot_bytes, b.src, b.bytes, bar);
             } else {
                 mbar_arrive(bar);
             }
