@@ -32,7 +32,7 @@ constexpr int kPipeHeaderReserve = 1024;    // mbarriers in front of the slots
 constexpr int kMaxBlockCols = 1024;         // columns per column block (32 fp32 accumulators per lane)
 constexpr long long kWaitCycles = 1LL << 31; // SM clock cycles (about a second) before an mbarrier wait gives up
 constexpr int kScanThreads = 256;
-constexpr int kScanItems = 8;               // rows per thread in the scan kernel
+constexpr int kScanItems = 4;               // rows per thread in the scan kernel (16: 2 % slower on r64, 8: 0.5 %)
 constexpr int kScanTile = kScanThreads * kScanItems;
 constexpr int kSmCount = 148;               // B200; only used to pick the chunk length
 constexpr unsigned kInvalidKey = 0xFFFFFFFFu;
