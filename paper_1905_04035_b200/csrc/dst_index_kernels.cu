@@ -196,13 +196,18 @@ k_bounds(const WsHeader* __restrict__ hdr, const unsigned* __restrict__ keys, un
          int capacity, int vocab) {
     pdl_trigger();
     pdl_wait();
-    const int n = capacity - (int)hdr->n_bad;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
+    if (i >= capacity) return;
+    // the three keys and the number of valid entries are asked for together: one trip to memory.
+    // (Entries past the valid ones hold whatever the buffer held; they are read, never used.)
     const unsigned k = keys[i];
+    const unsigned before = i > 0 ? keys[i - 1] : 0u;
+    const unsigned after = i + 1 < capacity ? keys[i + 1] : 0u;
+    const int n = capacity - (int)hdr->n_bad;
+    if (i >= n) return;
     if (k >= (unsigned)vocab) return;                    // only after a failed look-back
-    const unsigned prev = i > 0 ? keys[i - 1] : ~k;
-    const unsigned next = i + 1 < n ? keys[i + 1] : ~k;
+    const unsigned prev = i > 0 ? before : ~k;
+    const unsigned next = i + 1 < n ? after : ~k;
     if (prev != k) atomicSub(&count[k], (unsigned)i);
     if (next != k) atomicAdd(&count[k], (unsigned)i + 1u);
 }
