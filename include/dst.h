@@ -217,9 +217,12 @@ int dst_densify_concat_host(const dst_slice_t* slices, int32_t R, int64_t d, int
  * (dst_workspace_bytes(plan.n_slice_rows, plan.n_slices, d, vocab, opts) when plan.converts != 0).
  *
  * dst_accumulate enqueues the work on `stream`:
- *   - dense output  -> out_dense [vocab, d] in opts->out_type.  The dense gradients are added left to
- *     right in fp32, then the slices are densified onto that sum in one pass (dst_densify_concat
- *     with out_dense as its dense partner), so the value rows cross the memory bus once.
+ *   - dense output  -> out_dense [vocab, d] in opts->out_type.  The dense gradients are added in fp32
+ *     in the order given, eight tensors per pass (with more than eight the running sum passes
+ *     through out_dense, in opts->out_type, between passes); a gradient that is out_dense itself is
+ *     taken first, so that it is read before the first pass overwrites it.  Then the slices are
+ *     densified onto that sum in one pass (dst_densify_concat with out_dense as its dense partner),
+ *     so the value rows cross the memory bus once.
  *     `result` (optional) is written only when slices were converted (plan.converts != 0).
  *   - slices output -> out_indices [out_rows], out_values [out_rows, d]: the concatenation.  Needs
  *     out_capacity_rows >= plan.out_rows, and value_type == out_type when a dense gradient is

@@ -1,17 +1,18 @@
 """Oracle for the gradient-accumulation strategies of the paper.  TEST INFRASTRUCTURE ONLY.
 
-Follows the paper's two algorithms step by step, in NumPy, with fp64 sums:
+What a list of gradients of one variable accumulates to, in NumPy, with fp64 sums:
 
-* Algorithm 1 (Section 3), the stock strategy: fewer than two gradients pass through; all-dense
-  gradients are summed; anything else is turned into IndexedSlices (a dense [vocab, d] tensor becomes
-  ``vocab`` slices, row v carrying index v, as Section 3 describes) and concatenated -- a gather.
-* Algorithm 2 (Section 6), the proposed strategy: one more branch before the gather -- if at least
-  one gradient is dense, every gradient is converted to a dense tensor and the tensors are summed.
-* Listing 1 (Section 4), Horovod's ``sparse_as_dense``: every IndexedSlices gradient is converted to a
-  dense tensor before accumulation, after which Algorithm 1 only ever sees dense tensors.
+* the stock rule (Section 3, Algorithm 1): a list of fewer than two gradients is handed on unchanged;
+  a list of dense tensors only is summed; any other list is turned into IndexedSlices (a dense
+  [vocab, d] tensor becomes ``vocab`` slices, row v carrying index v, as Section 3 describes) and
+  concatenated -- a gather;
+* the proposed rule (Section 6, Algorithm 2): the same, except that a mixed list holding at least one
+  dense tensor is converted to dense tensors and summed instead of gathered;
+* Horovod's ``sparse_as_dense`` (Section 4, Listing 1): every IndexedSlices gradient is made dense
+  before the stock rule sees the list, which can then only pass through or sum.
 
-``conv_to_tensor`` of an IndexedSlices gradient is the scatter-sum of ``oracle.densify`` (duplicates
-add up).  Nothing here is imported by the CUDA library or its binding.
+Making IndexedSlices dense is the scatter-sum of ``oracle.densify`` (duplicates add up).  Nothing here
+is imported by the CUDA library or its binding.
 
 Pins: ``tests/test_accumulate_oracle.py`` (hand-worked example, strategy-independence of the
 accumulated value, the paper's row counts, pass-through identity, library sum).
@@ -42,48 +43,51 @@ class Grad:
 
 @dataclasses.dataclass
 class Accumulated:
-    branch: str               # which line of the algorithm produced it
+    branch: str               # which rule produced it
     grad: Optional[Grad]      # None for an empty input; dense values are float64 sums
 
 
-def conv_to_tensor(g: Grad, d: int, vocab: int) -> np.ndarray:
-    """``tf.convert_to_tensor`` of Listing 1: a dense tensor is itself, IndexedSlices are scatter-summed."""
+def densified(g: Grad, d: int, vocab: int) -> np.ndarray:
+    """The gradient as a dense fp64 [vocab, d] array: a dense tensor is itself, IndexedSlices are scatter-summed."""
     if g.is_dense:
         return np.asarray(g.values, np.float64).reshape(vocab, d)
     return dst_oracle.densify([np.asarray(g.indices)], [np.asarray(g.values, np.float32)], d, vocab).acc
 
 
 def as_slices(g: Grad, d: int, vocab: int, index_dtype) -> Grad:
-    """Algorithm 1's gather branch sees everything as IndexedSlices: a dense tensor names every row once."""
+    """The gradient as IndexedSlices: a dense tensor names every row once (Section 3)."""
     if not g.is_dense:
         return g
     return Grad(np.asarray(g.values).reshape(vocab, d), np.arange(vocab, dtype=index_dtype))
 
 
+def rule(n: int, n_dense: int, strategy: str) -> str:
+    """Which rule a list of ``n`` gradients, ``n_dense`` of them dense, falls under."""
+    if n < 2:
+        return PASS_THROUGH
+    if n_dense == n:
+        return REDUCE
+    if strategy == PROPOSED and n_dense > 0:
+        return CONVERT_AND_REDUCE
+    return GATHER
+
+
 def accumulate(grads: Sequence[Grad], d: int, vocab: int, strategy: str = PROPOSED,
                index_dtype=np.int64) -> Accumulated:
+    if strategy not in (STOCK, PROPOSED, SPARSE_AS_DENSE):
+        raise ValueError(strategy)
     grads = list(grads)
     if strategy == SPARSE_AS_DENSE:
-        # Listing 1: convert each IndexedSlices gradient first, then the stock algorithm runs
-        grads = [g if g.is_dense else Grad(conv_to_tensor(g, d, vocab)) for g in grads]
-    elif strategy not in (STOCK, PROPOSED):
-        raise ValueError(strategy)
-    # line 1-2 of both algorithms
-    if len(grads) < 2:
-        return Accumulated(PASS_THROUGH, grads[0] if grads else None)
-    # line 3-4 of both algorithms
-    if all(g.is_dense for g in grads):
+        grads = [g if g.is_dense else Grad(densified(g, d, vocab)) for g in grads]
+    how = rule(len(grads), sum(g.is_dense for g in grads), strategy)
+    if how == PASS_THROUGH:
+        return Accumulated(how, grads[0] if grads else None)
+    if how in (REDUCE, CONVERT_AND_REDUCE):
         total = np.zeros((vocab, d), np.float64)
         for g in grads:
-            total += np.asarray(g.values, np.float64).reshape(vocab, d)
-        return Accumulated(REDUCE, Grad(total))
-    # Algorithm 2 only: any dense gradient -> convert all, reduce
-    if strategy == PROPOSED and any(g.is_dense for g in grads):
-        total = np.zeros((vocab, d), np.float64)
-        for g in grads:
-            total += conv_to_tensor(g, d, vocab)
-        return Accumulated(CONVERT_AND_REDUCE, Grad(total))
-    # last branch of both: gather (concatenation of IndexedSlices in the order given)
+            total += densified(g, d, vocab)
+        return Accumulated(how, Grad(total))
+    # gather: the concatenation of the IndexedSlices forms, in the order given
     parts: List[Grad] = [as_slices(g, d, vocab, index_dtype) for g in grads]
     indices = np.concatenate([np.asarray(p.indices).astype(index_dtype) for p in parts])
     values = np.concatenate([np.asarray(p.values).reshape(-1, d) for p in parts], axis=0)

@@ -25,16 +25,15 @@ static bool opts_ok(const dst_opts_t* o) {
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static int sm_count() {
-    static int cached = 0;
-    if (cached == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-            cached = n;
-        else
-            return kSmCount;
-    }
-    return cached;
+    // asked of the runtime once per device ordinal
+    constexpr int kDevices = 64;
+    static std::atomic<int> cached[kDevices];
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return kSmCount;
+    if (dev >= 0 && dev < kDevices && (n = cached[dev].load()) > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return kSmCount;
+    if (dev >= 0 && dev < kDevices) cached[dev].store(n);
+    return n;
 }
 
 static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
@@ -442,11 +441,20 @@ int dst_accumulate(const dst_grad_t* grads, int32_t n, int64_t d, int64_t vocab,
     if (p.n_dense == 1 && p.n_slices > 0) {
         for (int i = 0; i < n; ++i) if (grads[i].kind == DST_GRAD_DENSE) partner = grads[i].values;
     } else if (p.n_dense >= 1) {
+        // The dense gradients in the order given, except that a gradient out_dense aliases goes first: the
+        // running sum lands in out_dense after every kSumFanIn tensors, which must not happen before that
+        // gradient has been read.
         SumParams sp{};
         sp.out = out_dense; sp.n_elems = n_elems; sp.vector_ok = aligned16(out_dense);
         bool first = true;
-        for (int i = 0; i < n; ++i) {
-            if (grads[i].kind != DST_GRAD_DENSE) continue;
+        int n_aliased = 0;
+        for (int i = 0; i < n; ++i)
+            if (grads[i].kind == DST_GRAD_DENSE && grads[i].values == out_dense) ++n_aliased;
+        if (n_aliased > kSumFanIn) return DST_ERR_INVALID_ARG;       // they would not all be read before the first write
+        for (int pos = n_aliased ? -n : 0; pos < n; ++pos) {
+            // first round (pos < 0): the gradients that are out_dense itself; second round: all others
+            const int i = pos < 0 ? pos + n : pos;
+            if (grads[i].kind != DST_GRAD_DENSE || (grads[i].values == out_dense) != (pos < 0)) continue;
             sp.src[sp.k++] = grads[i].values;
             sp.vector_ok = sp.vector_ok && aligned16(grads[i].values);
             if (sp.k == kSumFanIn) {

@@ -661,14 +661,16 @@ template <typename VT, typename OT>
 __global__ void __launch_bounds__(256)
 k_reduce_rows_scalar(const MainArgs a) {
     const long long total = (long long)a.vocab * a.d;
-    if (blockIdx.x == 0 && threadIdx.x == 0 && a.result) a.result->status = a.hdr->status;
+    const int status = *reinterpret_cast<volatile int*>(&a.hdr->status);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && a.result) a.result->status = status;
+    if (status == DST_ERR_TIMEOUT) return;     // a wait gave up in an earlier kernel: the tables are not to be trusted
     const OT* din = static_cast<const OT*>(a.dense_in);
     OT* out = static_cast<OT*>(a.out);
     for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
         const int v = (int)(e / a.d);
         const long long c = e - (long long)v * a.d;
-        const int beg = a.offsets[v], end = a.offsets[v + 1];
-        if (beg == end && !a.apply) { out[e] = din ? din[e] : OT(0.f); continue; }
+        const int beg = max(a.offsets[v], 0), end = min(a.offsets[v + 1], a.n_total);
+        if (beg >= end && !a.apply) { out[e] = din ? din[e] : OT(0.f); continue; }
         float acc = 0.f;
         for (int j = beg; j < end; ++j) {
             unsigned p = a.perm[j];

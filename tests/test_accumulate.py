@@ -136,7 +136,7 @@ def test_accumulate_exact_on_small_integers_and_strategy_independent(strategy):
     else:
         n = plan["out_rows"]
         assert n == 2 * vocab + 900 + 5000 + 33
-        back = ao.conv_to_tensor(ao.Grad(out_val[:n].cpu().numpy(), out_idx[:n].cpu().numpy()), d, vocab)
+        back = ao.densified(ao.Grad(out_val[:n].cpu().numpy(), out_idx[:n].cpu().numpy()), d, vocab)
         assert np.array_equal(back, want)
 
 
@@ -151,7 +151,7 @@ def test_accumulate_bf16_int32_and_unaligned_rows():
     plan, _, out_idx, out_val, _, _ = run_gpu(grads, d, vocab, dst.DST_ACC_STOCK, value_kind="bf16", index_dtype=torch.int32)
     n = plan["out_rows"]
     assert n == 2 * vocab + 450 and out_idx.dtype == torch.int32
-    back = ao.conv_to_tensor(ao.Grad(widen(out_val[:n]).astype(np.float32), out_idx[:n].cpu().numpy()), d, vocab)
+    back = ao.densified(ao.Grad(widen(out_val[:n]).astype(np.float32), out_idx[:n].cpu().numpy()), d, vocab)
     assert np.array_equal(back, want)
 
 
@@ -170,6 +170,30 @@ def test_accumulate_in_place_and_capacity_check():
     small_v = torch.empty(10, d, device=dev)
     with pytest.raises(dst.DstError):
         dst.dst_accumulate([dense, sl], d, vocab, dst.DST_ACC_STOCK, out_indices=small_i, out_values=small_v)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("spec, alias", [(["D"] * 9 + [500], 8), (["D"] * 17, 16), (["D"] * 17, 3),
+                                         (["D"] * 12 + [100, 40], 11), (["D"] * 9, 0)])
+def test_accumulate_out_is_a_late_dense_gradient(spec, alias):
+    """out_dense may be one of the dense gradients, whatever its place in the list: with more than eight
+    dense gradients the sum runs in several passes through out_dense, and the aliased gradient must
+    have been read before the first pass lands.  Small integers: exact in any order."""
+    vocab, d = 600, 32
+    grads = make_list(spec, vocab, d, 21, integers=True)
+    want = ao.accumulate(grads, d, vocab, ao.PROPOSED).grad.values
+    dev = "cuda"
+    tg = [torch.from_numpy(g.values).to(dev) if g.is_dense
+          else (torch.from_numpy(g.indices).to(dev), torch.from_numpy(g.values).to(dev)) for g in grads]
+    n_rows = sum(s for s in spec if s != "D")
+    n_sl = sum(1 for s in spec if s != "D")
+    ws = torch.empty(max(256, dst.dst_workspace_bytes(n_rows, max(n_sl, 1), d, vocab)), dtype=torch.uint8, device=dev)
+    dst.dst_accumulate(tg, d, vocab, dst.DST_ACC_PROPOSED, out_dense=tg[alias], workspace=ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(widen(tg[alias]), want)
+    for k, g in enumerate(grads):                  # every other gradient is untouched
+        if g.is_dense and k != alias:
+            assert np.array_equal(tg[k].cpu().numpy(), g.values)
 
 
 @pytest.mark.gpu

@@ -55,11 +55,11 @@ def test_accumulated_value_does_not_depend_on_the_strategy():
         np.add.at(direct, g.indices, g.values.astype(np.float64))     # library scatter-add
     assert np.array_equal(ref, direct)
     st = ao.accumulate(grads, d, vocab, ao.STOCK).grad
-    assert np.array_equal(ao.conv_to_tensor(st, d, vocab), ref)
+    assert np.array_equal(ao.densified(st, d, vocab), ref)
     assert np.array_equal(ao.accumulate(grads, d, vocab, ao.SPARSE_AS_DENSE).grad.values, ref)
     # all-sparse input: the gathered slices densify to what sparse_as_dense reduces to
     sp = ao.accumulate(grads[1:], d, vocab, ao.STOCK).grad
-    assert np.array_equal(ao.conv_to_tensor(sp, d, vocab), ao.accumulate(grads[1:], d, vocab, ao.SPARSE_AS_DENSE).grad.values)
+    assert np.array_equal(ao.densified(sp, d, vocab), ao.accumulate(grads[1:], d, vocab, ao.SPARSE_AS_DENSE).grad.values)
 
 
 def test_gather_row_count_is_the_papers_accounting():
