@@ -80,10 +80,14 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         if (slices[r].n_rows > 0 && !aligned16(slices[r].values)) vector_ok = false;
 
     const unsigned* perm = pos[L.passes & 1];
-    bool compact = false;
-    const bool small = n_total <= kFrontMaxRows && vocab <= 65536 && R <= kHistSlices;
+    bool compact = false, overlap = false;
+    // Small input with no more input rows than vocabulary rows (and rows the vector kernels can take): one cluster
+    // kernel does the whole index side.  Most output rows are then named by nobody: the tables list the named
+    // rows only, and the row-reduction kernel, running beside the index cluster, gives the other rows their
+    // dense_in row (or zeros, or the dense part of the SGD step) while the index work is under way.  In place
+    // there is nothing to do for those rows.
+    const bool small = n_total <= kFrontMaxRows && vocab <= 65536 && R <= kHistSlices && vector_ok && n_total <= vocab;
     if (small) {
-        // small input: one cluster kernel does the whole index side and clears its own tables
         FrontParams fp;
         memset(&fp.P, 0, sizeof fp.P);
         fp.P.n = R;
@@ -92,24 +96,17 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
             fp.P.s[i] = SliceEntry{slices[i].indices, slices[i].values, (long long)start, (long long)slices[i].n_rows};
             start += slices[i].n_rows;
         }
-        fp.hdr = hdr; fp.tab = tab; fp.perm = pos[0]; fp.offsets = offsets; fp.heavy = heavy;
-        fp.unique_rows = unique_rows; fp.counts_out = counts; fp.result = result; fp.batches = batches;
-        fp.node_cnt = nodecnt; fp.vocab = vocab; fp.n_total = int(n_total); fp.vocab_pad = int(L.vocab_pad);
-        fp.chunk = L.chunk; fp.batch_units = L.batch_units; fp.batch_max = int(L.batch_max);
+        fp.hdr = hdr; fp.tab = tab; fp.perm = pos[0]; fp.heavy = heavy;
+        fp.unique_rows = unique_rows; fp.counts_out = counts; fp.result = result;
+        fp.node_cnt = nodecnt; fp.vocab = vocab; fp.n_total = int(n_total);
+        fp.chunk = L.chunk; fp.batch_units = L.batch_units; fp.batches = batches; fp.batch_max = int(L.batch_max);
         fp.nodecnt_words = int((L.off_batches - L.off_nodecnt) / 4);
-        // No more input rows than vocabulary rows: most output rows are plain copies of dense_in.  Extra
-        // clusters of the same launch write out = dense_in (or zeros) for every row while the first cluster
-        // does the index work; the row-reduction kernel then visits only the rows that were named (and
-        // reads and writes those a second time).  In place there is nothing to copy.
-        compact = vector_ok && n_total <= vocab;
-        fp.compact = compact ? 1 : 0;
+        compact = true;
+        overlap = apply ? dense_in != nullptr : out != dense_in;
         fp.urow = reinterpret_cast<int*>(ws + L.off_urow);
         fp.uoff = reinterpret_cast<int*>(ws + L.off_uoff);
-        fp.copy_src = dense_in; fp.copy_dst = out;
-        fp.copy_bytes = int64_t(vocab) * d * int64_t(dtype_size(opts->out_type));
-        fp.copy_clusters = compact && out != dense_in ? (sm_count() - kClusterCtas) / kClusterCtas : 0;
-        fp.copy_apply = apply ? 1 : 0; fp.copy_lr = lr;
-        if (apply && !dense_in) fp.copy_clusters = 0;   // nothing to take from the rows nobody names
+        fp.bitmap = reinterpret_cast<unsigned*>(ws + L.off_bitmap);
+        fp.bitmap_words = L.bitmap_words;
         if (launch_front_cluster(opts->index_type, fp, stream) != cudaSuccess) return DST_ERR_CUDA;
         ++g_launches;
         perm = pos[0];
@@ -163,6 +160,10 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     a.chunk_max = int(L.chunk_max); a.upper_max = int(L.upper_max);
     a.W = a.ncb = a.slot_bytes = a.n_slots = 0;   // set by the launcher
     a.compact = compact ? 1 : 0;
+    a.overlap = overlap ? 1 : 0;
+    a.bitmap = reinterpret_cast<const unsigned*>(ws + L.off_bitmap);
+    a.bitmap_words = L.bitmap_words;
+    a.copy_rows = 8;     // set by the launcher
     a.apply = apply ? 1 : 0; a.lr = lr;
     a.urow = reinterpret_cast<const int*>(ws + L.off_urow);
     a.uoff = reinterpret_cast<const int*>(ws + L.off_uoff);

@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <utility>
 
 #include "dst.h"
@@ -58,8 +59,13 @@ struct WsHeader {          // zeroed at the start of every call
     int n_batches;         // light work items (row batches)
     unsigned int scan_ticket;
     unsigned int scan_done;
+    unsigned int copy_counter;   // small-input path: copy work items handed out
+    int tables_ready;            // ... set by the index cluster once every table and this header are written
+    int reserved[2];
+    int bitmap_ready[kClusterCtas];   // ... CTA r of the index cluster has written its copy of the named-row bitmap
 };
-static_assert(sizeof(WsHeader) == 72, "header layout");
+static_assert(sizeof(WsHeader) == 120, "header layout");
+constexpr int kHeaderWordsBeforeFlags = (120 - 4 * kClusterCtas) / 4;   // words the index cluster's first CTA clears
 
 struct SliceEntry {        // one IndexedSlices object of the (virtual) concatenation
     const void* indices;
@@ -98,7 +104,8 @@ struct Layout {
     int R, chunk, passes, batch_units;
     int64_t n_tiles, vocab_pad, heavy_max, chunk_max, upper_max, batch_max;
     size_t off_header, off_count, off_digit, off_desc, off_nodecnt, off_batches, off_scandesc, zero_bytes;
-    size_t off_offsets, off_keys[2], off_pos[2], off_tab, off_heavy, off_partials, off_urow, off_uoff;
+    size_t off_offsets, off_keys[2], off_pos[2], off_tab, off_heavy, off_partials, off_urow, off_uoff, off_bitmap;
+    int bitmap_words;        // 32-bit words of the named-row bitmap (small-input path), 0 when that path cannot apply
     size_t total;
 };
 
@@ -109,7 +116,7 @@ struct MainArgs {
     const unsigned* perm;
     const SliceEntry* tab;
     const HeavyInfo* heavy;
-    const int2* batches;   // per row batch: first row + 1 (0: empty batch), last row + 1; `compact`: numbers in urow[]
+    const int2* batches;   // per row batch: first row + 1, last row + 1 (0: empty batch); `compact`: ranks among the named rows
     const int* urow;       // compact: the named rows, ascending
     const int* uoff;       // compact: first entry of each named row in perm[], then the number of entries
     unsigned* node_cnt;
@@ -130,7 +137,14 @@ struct MainArgs {
     int n_slots;
     int apply;       // 1: `out` holds a weight and gets the SGD step (fp32 only), see dst_densify_apply_sgd
     float lr;        // learning rate of that step
-    int compact;     // out already holds dense_in (or zeros) everywhere: the row batches list only the named rows
+    int compact;     // the row batches list only the named rows (urow / uoff); the others are not this item list's business
+    // Overlapped small-input path: the kernel starts beside the index cluster.  Until tables_ready it gives the rows
+    // nobody names their dense_in row (copy items of copy_rows consecutive rows, named ones skipped by the bitmap),
+    // then it takes the named rows, then whatever copy items are left.
+    int overlap;
+    int copy_rows;              // rows per copy item: 8, 16 or 32 (a divisor of 32)
+    const unsigned* bitmap;     // kClusterCtas interleaved copies, see Layout::off_bitmap
+    int bitmap_words;
 };
 
 // How the row-reduction kernel cuts rows into column blocks and shared memory into slots.
@@ -163,7 +177,11 @@ inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab, i
     const int64_t max_chunk = kMaxChunkRows;
     while (c < max_chunk && c * 2 <= share) c *= 2;
     L.batch_units = int(share < 8 ? 8 : (share > kMaxBatchUnits ? kMaxBatchUnits : share));
-    L.batch_max = (vocab + n_rows) / L.batch_units + 2;
+    {
+        int pow2 = 8;                                     // the small-input path cuts items of the power of two below batch_units
+        while (pow2 * 2 <= L.batch_units) pow2 *= 2;
+        L.batch_max = (vocab + n_rows) / pow2 + 2;
+    }
     L.chunk = c;
     int bits = 0;
     while (bits < 31 && (int64_t(1) << bits) < vocab) ++bits;   // keys are < vocab <= 2^bits
@@ -195,6 +213,9 @@ inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab, i
         L.off_urow = take(size_t(cap) * 4);
         L.off_uoff = take(size_t(cap) * 4);
     }
+    // named-row bitmap of the small-input path: one copy per CTA of the index cluster, word w of copy r at [w * 8 + r]
+    L.bitmap_words = (n_rows <= kFrontMaxRows && vocab <= 65536) ? int((vocab + 31) / 32) : 0;
+    L.off_bitmap = take(size_t(L.bitmap_words) * kClusterCtas * 4);
     L.off_partials = take(size_t(L.chunk_max + L.upper_max) * size_t(d) * 4);
     L.total = o;
     return L;
@@ -223,24 +244,18 @@ struct FrontParams {
     WsHeader* hdr;
     SliceEntry* tab;
     unsigned* perm;
-    int* offsets;
     HeavyInfo* heavy;
     void* unique_rows;
     int* counts_out;
     dst_result_t* result;
-    int2* batches;
     unsigned* node_cnt;
+    int2* batches;
     long long vocab;
-    int n_total, vocab_pad, chunk, batch_units, batch_max, nodecnt_words;
-    int compact;               // list only the named rows in the row batches (and in urow / uoff)
-    int* urow;
-    int* uoff;
-    const void* copy_src;      // with copy_clusters > 0: dense_in, or nullptr to fill out with zeros
-    void* copy_dst;            // out
-    long long copy_bytes;      // vocab * d * sizeof(out element), a multiple of 16
-    int copy_clusters;         // extra clusters that fill out while the first one does the index work
-    int copy_apply;            // 1: the extra clusters take the dense part of the SGD step, out -= copy_lr * dense_in (fp32)
-    float copy_lr;
+    int n_total, chunk, batch_units, batch_max, nodecnt_words;
+    int* urow;                 // the named rows, ascending
+    int* uoff;                 // first entry of each named row in perm[], then the number of entries
+    unsigned* bitmap;          // named-row bitmap, written early for the row-reduction kernel running beside this one
+    int bitmap_words;
 };
 cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStream_t stream);
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
@@ -274,6 +289,19 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+// The opt-in to a kernel's dynamic shared memory size is made once per device and kernel (and again when a
+// larger size is asked for), not on every call.  One cache object per kernel instantiation.
+struct SmemOptIn { std::atomic<int> bytes[64]; };
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, size_t bytes, SmemOptIn& cache) {
+    int dev = -1;
+    const bool cached = cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64;
+    if (cached && cache.bytes[dev].load() >= (int)bytes) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess && cached) cache.bytes[dev].store((int)bytes);
+    return e;
 }
 
 // ---- device helpers ---------------------------------------------------------

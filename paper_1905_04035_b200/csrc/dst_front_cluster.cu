@@ -1,25 +1,32 @@
 // Index side of densify for small inputs, in one kernel: a thread-block cluster of kClusterCtas
-// CTAs validates the indices, sorts them (two stable 8-bit radix passes), takes the run lengths and
-// scans them into every table the row-reduction kernel needs.
+// CTAs validates the indices, sorts them (two stable 8-bit radix passes) and walks the sorted
+// order once to produce every table the row-reduction kernel needs.
 //
 // Why a cluster: for a Transformer batch of a few thousand tokens (the paper's Section 3 setting)
 // the index work is pure latency.  Spread over separate kernels it costs more launches than work;
 // in one CTA it is bound by one SM's instruction rate.  Eight CTAs on eight SMs share the work and
 // exchange what they must through distributed shared memory and cluster barriers:
 //   - the per-digit counts of each CTA (to place a CTA's entries behind those of the CTAs before it),
-//   - the entries themselves: pass 0 scatters each packed entry (key << 16 | position) into the
+//   - the entries themselves: each pass scatters every packed entry (key << 16 | position) into the
 //     shared memory of the CTA that owns that part of the sorted order,
-//   - count[v], kept in shared memory, a slice of the vocabulary per CTA,
-//   - the per-CTA sums of the final scan.
+//   - one summary per CTA of the segmented scan over the sorted entries.
 // Nothing spins: the only waits are cluster barriers that every thread of every CTA reaches the same
-// number of times.  The kernel also clears the few global tables that must start at zero, so this
-// path needs no memset.
+// number of times.
 //
+// The row-reduction kernel is launched as a programmatic dependent of this one and runs beside it on
+// the other SMs, moving most of the bytes of the call meanwhile, so every access this kernel makes to
+// global memory queues behind that traffic.  Hence the shape of the kernel: global memory is read once
+// (the indices) and written at two points only -- a bitmap of the named rows as soon as the indices are
+// validated (the rows outside it only need their dense_in row, which the other kernel copies while the
+// sort is still running), and all tables in one burst at the end, followed by one flag.  Everything in
+// between lives in shared memory.  The header with the flags is cleared before the dependent launch is
+// released.
+//
+// The tables list the named rows only (by rank u among them: row number urow[u], first entry uoff[u]),
+// which is why this path is taken only when there are no more input rows than vocabulary rows.
 // Limits: n_total <= kFrontMaxRows (positions fit 16 bits), vocab <= 65536 (keys fit 16 bits),
 // R <= kHistSlices (the slice table travels as a kernel parameter).
 #include <cooperative_groups.h>
-
-#include <atomic>
 
 #include "dst_common.cuh"
 
@@ -32,445 +39,416 @@ struct FrontArgs {
     WsHeader* hdr;
     SliceEntry* tab;
     unsigned* perm;
-    int* offsets;
     HeavyInfo* heavy;
     void* unique_rows;
     int* counts_out;
     dst_result_t* result;
-    int2* batches;
     int* urow;
     int* uoff;
-    int compact;
     unsigned* node_cnt;
+    int2* batches;             // light work items: ranks (+ 1) of the first and last named row that start in each
+    unsigned* bitmap;          // [bitmap_words][kClusterCtas]: this CTA's copy of the named-row bitmap at [w * 8 + rank]
     long long vocab;
-    int n_total, vocab_pad, chunk, batch_units, batch_max, nodecnt_words;
+    int n_total, chunk_log, batch_log, batch_max, nodecnt_words, bitmap_words;
     int lw;                    // entries per warp (multiple of 32); a CTA's slice of the sorted order holds 32 * lw
-    int rpt;                   // vocabulary rows per thread in the scan; a CTA's slice of count[] holds 1024 * rpt
-    const uint4* copy_src;     // clusters after the first: out = dense_in (or zeros), 16 bytes per thread and step
-    uint4* copy_dst;
-    long long copy_vecs;
-    int copy_apply;            // out -= copy_lr * dense_in instead of out = dense_in (fp32 tensors)
-    float copy_lr;
 };
 
 constexpr int kFrontWarps = kFrontThreads / 32;
 constexpr int kFrontGroups = 8;       // groups of 32 entries per warp, at most (kFrontMaxRows / 256 / 32)
-constexpr int kFrontRpt = 8;          // rows per thread, at most (65536 / 8192)
+constexpr int kFrontParts = 4;        // the warps of a CTA in four parts of eight for the digit prefix
 
-// one group of 32 entries: add it to the warp's running digit counters and return this lane's
-// rank among the warp's entries so far with the same digit (wh: this warp's 256 counters)
-__device__ __forceinline__ unsigned rank_step(unsigned short* wh, bool valid, unsigned dg, int lane) {
-    const unsigned m = match_digit(dg & 255u, valid);
-    const int leader = valid ? __ffs(m) - 1 : lane;
-    unsigned pre = 0;
-    if (valid && lane == leader) { pre = wh[dg]; wh[dg] = (unsigned short)(pre + __popc(m)); }
-    pre = __shfl_sync(0xFFFFFFFFu, pre, leader);
-    __syncwarp();
-    return pre + __popc(m & ((1u << lane) - 1u));
+// A note on the style of this file.  The code of this kernel is fetched cold on every launch, through a
+// memory system that the row-reduction kernel keeps saturated meanwhile, and is executed once: its
+// running time follows the bytes of straight-line code more than the instructions executed.  So loops
+// stay rolled (#pragma unroll 1), per-entry state lives in shared memory instead of register arrays,
+// and what is needed at several places exists once.
+
+// Lanes of the warp whose 8-bit digit equals this lane's, among the lanes with `valid` set.
+__device__ __forceinline__ unsigned match_digit_rolled(unsigned dg, bool valid) {
+    unsigned m = __ballot_sync(0xFFFFFFFFu, valid);
+#pragma unroll 1
+    for (int b = 0; b < 8; ++b) {
+        const bool bit = (dg >> b) & 1u;
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, bit);
+        m &= bit ? bal : ~bal;
+    }
+    return m;
 }
 
-// After every warp has counted its digits into wh[w][d]: turn the counts into the sorted position
-// of the first entry of (digit d, this CTA, warp w).  One cluster barrier inside.  Returns the
-// number of entries over the whole cluster.
-__device__ __forceinline__ unsigned cluster_bases(cg::cluster_group& cluster, unsigned short (*wh)[256],
-                                                  unsigned* cta_tot, unsigned* s_warp_tot, unsigned* s_total) {
-    const int lane = lane_id(), warp = warp_id();
-    const unsigned rank = cluster.block_rank();
-    unsigned tot = 0;
-    if (threadIdx.x < 256) {
-#pragma unroll 8
-        for (int w = 0; w < kFrontWarps; ++w) { unsigned t = wh[w][threadIdx.x]; wh[w][threadIdx.x] = (unsigned short)tot; tot += t; }
-        cta_tot[threadIdx.x] = tot;
-    }
-    cluster.sync();                                   // every CTA's per-digit totals are in place
-    unsigned before = 0, all = 0;
-    if (threadIdx.x < 256) {
-#pragma unroll
-        for (unsigned c = 0; c < (unsigned)kClusterCtas; ++c) {
-            const unsigned t = cluster.map_shared_rank(cta_tot, c)[threadIdx.x];
-            if (c < rank) before += t;
-            all += t;
-        }
-    }
-    unsigned inc = all;                               // exclusive scan of the digit totals over the 256 digits
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { unsigned t = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t; }
-    if (lane == 31 && warp < 8) s_warp_tot[warp] = inc;
-    __syncthreads();
-    if (threadIdx.x < 256) {
-        unsigned base = inc - all + before;
-        for (int w = 0; w < warp; ++w) base += s_warp_tot[w];
-#pragma unroll 8
-        for (int w = 0; w < kFrontWarps; ++w) wh[w][threadIdx.x] = (unsigned short)(wh[w][threadIdx.x] + base);
-        if (threadIdx.x == 255) *s_total = base - before + all;
-    }
-    __syncthreads();
-    return *s_total;
-}
+struct DigitScratch {
+    unsigned short wh[kFrontWarps][256];      // per warp and digit: count, then exclusive prefix inside the warp's part
+    unsigned short part_tot[kFrontParts][256];
+    unsigned cta_tot[256];                    // this CTA's entries per digit (read by the other CTAs)
+    unsigned base[kFrontParts][256];          // sorted position of the first entry of (digit, this CTA, part)
+    unsigned warp_tot[8];
+    unsigned total;
+};
 
-struct Sum6 { int v[6]; };   // 0 offset, 1 unique, 2 heavy rows, 3 chunks, 4 upper nodes, 5 units of the light work items
+// ---- the segmented scan over the sorted entries --------------------------------------------------
+// What a stretch of consecutive sorted entries knows about the rows (runs of equal keys) it touches.
+// A row is accounted for where its last entry (its tail) lies; its length needs the position of its
+// first entry (its head), which may lie in an earlier stretch: such a tail stays open (`bt`) until
+// the stretches are combined.  At most one tail of a stretch can be open: the first, when no head
+// comes before it.
+struct Seg {
+    int nt;     // tails: rows that end in the stretch
+    int nh;     // of those with a known length: heavy rows,
+    int nc;     //   their chunks,
+    int nu;     //   their upper combine-tree nodes,
+    int un;     // of the rows with a known length: units of light work (entries + 1; a heavy row counts 1)
+    int mx;     // longest known row
+    int lh;     // position of the last head in the stretch, -1: none
+    int bt;     // position of the open tail, -1: none
+};
+__device__ __forceinline__ Seg seg_identity() { return Seg{0, 0, 0, 0, 0, 0, -1, -1}; }
+// Chunks and upper tree nodes of a heavy row, packed (nodes << 16 | chunks; a row has at most 4096 chunks).
+// Out of line on purpose: heavy rows are few, and the code of this kernel is fetched cold on every
+// launch, through a memory system that the row-reduction kernel keeps busy, so every kilobyte of
+// straight-line code on the common path is paid for in time.
+__device__ __noinline__ unsigned heavy_shape(int count, int chunk_log) {
+    const int n = (count + (1 << chunk_log) - 1) >> chunk_log;
+    return ((unsigned)upper_nodes(n) << 16) | (unsigned)n;
+}
+__device__ __forceinline__ void seg_add_row(Seg& s, int count, int chunk_log) {
+    s.mx = max(s.mx, count);
+    s.un += row_units(count, 1 << chunk_log);
+    if (count > (1 << chunk_log)) {
+        const unsigned hs = heavy_shape(count, chunk_log);
+        s.nh += 1; s.nc += (int)(hs & 0xFFFFu); s.nu += (int)(hs >> 16);
+    }
+}
+// stretch A followed by stretch B
+__device__ __forceinline__ Seg seg_combine(const Seg& A, const Seg& B, int chunk_log) {
+    Seg r;
+    r.nt = A.nt + B.nt; r.nh = A.nh + B.nh; r.nc = A.nc + B.nc; r.nu = A.nu + B.nu; r.un = A.un + B.un;
+    r.mx = max(A.mx, B.mx);
+    if (B.bt >= 0 && A.lh >= 0) seg_add_row(r, B.bt - A.lh + 1, chunk_log);
+    r.bt = A.bt >= 0 ? A.bt : (A.lh < 0 ? B.bt : -1);
+    r.lh = B.lh >= 0 ? B.lh : A.lh;
+    return r;
+}
+__device__ __forceinline__ Seg seg_shfl_up(const Seg& s, int o) {
+    Seg t;
+    t.nt = __shfl_up_sync(0xFFFFFFFFu, s.nt, o); t.nh = __shfl_up_sync(0xFFFFFFFFu, s.nh, o);
+    t.nc = __shfl_up_sync(0xFFFFFFFFu, s.nc, o); t.nu = __shfl_up_sync(0xFFFFFFFFu, s.nu, o);
+    t.un = __shfl_up_sync(0xFFFFFFFFu, s.un, o); t.mx = __shfl_up_sync(0xFFFFFFFFu, s.mx, o);
+    t.lh = __shfl_up_sync(0xFFFFFFFFu, s.lh, o); t.bt = __shfl_up_sync(0xFFFFFFFFu, s.bt, o);
+    return t;
+}
+__device__ __forceinline__ Seg seg_shfl(const Seg& s, int src) {
+    Seg t;
+    t.nt = __shfl_sync(0xFFFFFFFFu, s.nt, src); t.nh = __shfl_sync(0xFFFFFFFFu, s.nh, src);
+    t.nc = __shfl_sync(0xFFFFFFFFu, s.nc, src); t.nu = __shfl_sync(0xFFFFFFFFu, s.nu, src);
+    t.un = __shfl_sync(0xFFFFFFFFu, s.un, src); t.mx = __shfl_sync(0xFFFFFFFFu, s.mx, src);
+    t.lh = __shfl_sync(0xFFFFFFFFu, s.lh, src); t.bt = __shfl_sync(0xFFFFFFFFu, s.bt, src);
+    return t;
+}
+// inclusive scan over the lanes of a warp; `excl` receives the exclusive one
+__device__ __forceinline__ Seg seg_warp_scan(Seg v, Seg& excl, int chunk_log) {
+    const int lane = lane_id();
+#pragma unroll 1
+    for (int o = 1; o < 32; o <<= 1) {
+        const Seg t = seg_shfl_up(v, o);
+        if (lane >= o) v = seg_combine(t, v, chunk_log);
+    }
+    excl = seg_shfl_up(v, 1);
+    if (lane == 0) excl = seg_identity();
+    return v;
+}
 
 template <typename IT>
 __global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kFrontThreads, 1)
 k_front_cluster(const __grid_constant__ FrontArgs f) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    __shared__ unsigned short wh[kFrontWarps][256];
-    __shared__ unsigned cta_tot[256];
-    __shared__ unsigned s_warp_tot[8];
-    __shared__ unsigned s_total;
-    __shared__ int s_scan[kFrontWarps][6];
-    __shared__ int cta_sum[6];
-    __shared__ int s_before[6], s_grand[6];
-    __shared__ int s_maxseg[kFrontWarps];
-    pdl_trigger();
-    pdl_wait();
-
-    if (blockIdx.x >= (unsigned)kClusterCtas) {
-        // Not the index cluster: meanwhile give every output row its dense_in row (or zeros).  The rows
-        // that do get contributions are rewritten by the row-reduction kernel; for a batch of a few
-        // thousand tokens against a vocabulary of tens of thousands that is a small part of the rows,
-        // and this copy, most of the bytes of the whole operation, hides the index work entirely.
-        const long long stride = (long long)(gridDim.x - kClusterCtas) * kFrontThreads;
-        long long i = (long long)(blockIdx.x - kClusterCtas) * kFrontThreads + threadIdx.x;
-        if (f.copy_src && f.copy_apply) {
-            // the dense part of the SGD step for every row: weight -= lr * dense gradient
-            const float4* src = reinterpret_cast<const float4*>(f.copy_src);
-            float4* dst = reinterpret_cast<float4*>(f.copy_dst);
-            const float nlr = -f.copy_lr;
-            for (; i + 3 * stride < f.copy_vecs; i += 4 * stride) {
-                float4 g[4], w[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) { g[q] = __ldcs(src + i + q * stride); w[q] = __ldcs(dst + i + q * stride); }
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    __stcs(dst + i + q * stride, make_float4(fmaf(nlr, g[q].x, w[q].x), fmaf(nlr, g[q].y, w[q].y),
-                                                            fmaf(nlr, g[q].z, w[q].z), fmaf(nlr, g[q].w, w[q].w)));
-            }
-            for (; i < f.copy_vecs; i += stride) {
-                const float4 g = __ldcs(src + i), w = __ldcs(dst + i);
-                __stcs(dst + i, make_float4(fmaf(nlr, g.x, w.x), fmaf(nlr, g.y, w.y), fmaf(nlr, g.z, w.z), fmaf(nlr, g.w, w.w)));
-            }
-        } else if (f.copy_src) {
-            for (; i + 7 * stride < f.copy_vecs; i += 8 * stride) {
-                uint4 v[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) v[q] = __ldcs(f.copy_src + i + q * stride);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) __stcs(f.copy_dst + i + q * stride, v[q]);
-            }
-            for (; i < f.copy_vecs; i += stride) __stcs(f.copy_dst + i, __ldcs(f.copy_src + i));
-        } else {
-            for (; i < f.copy_vecs; i += stride) __stcs(f.copy_dst + i, make_uint4(0u, 0u, 0u, 0u));
-        }
-        return;
-    }
+    __shared__ DigitScratch dg;
+    __shared__ Seg s_warp_seg[kFrontWarps];     // per warp: its stretch
+    __shared__ Seg s_warp_pre[kFrontWarps];     // per warp: the stretch of the warps before it
+    __shared__ Seg s_cta_seg;                   // this CTA's stretch (read by the other CTAs)
+    __shared__ Seg s_before, s_grand;           // the stretch of the CTAs before this one / of all CTAs
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const int lane = lane_id(), warp = warp_id();
     const int S = 32 * f.lw;                         // entries of the sorted order this CTA owns
-    const int Vs = kFrontThreads * f.rpt;            // rows of count[] this CTA owns
-    unsigned* packed = reinterpret_cast<unsigned*>(dyn);                          // [S] key << 16 | position
-    unsigned* cnt = packed + S;                                                   // [Vs]
-    unsigned short* skey = reinterpret_cast<unsigned short*>(cnt + Vs);           // [S] sorted keys
+    const int ng = f.lw / 32;                        // groups of 32 entries per warp = entries per thread
+    // two buffers of packed entries (key << 16 | position; 0xFFFFFFFF: no entry): the passes go from one to the other
+    unsigned* buf0 = reinterpret_cast<unsigned*>(dyn);                            // [S]
+    unsigned* buf1 = buf0 + S;                                                    // [S]
+    unsigned short* rks = reinterpret_cast<unsigned short*>(buf1 + S);            // [S] rank of an entry among its warp's entries with the same digit
+    unsigned char* named = reinterpret_cast<unsigned char*>(rks + S);             // [32 * bitmap_words] 1: some valid entry names the row
     WsHeader* hdr = f.hdr;
     const int gt = rank * kFrontThreads + threadIdx.x;   // thread id in the cluster
     constexpr int kAllThreads = kClusterCtas * kFrontThreads;
 
-    // ---- clear what must start at zero
-    for (int i = threadIdx.x; i < Vs; i += kFrontThreads) cnt[i] = 0;
-    for (int i = gt; i < f.batch_max; i += kAllThreads) f.batches[i] = make_int2(f.compact ? 0x7FFFFFFF : 0, 0);
-    for (int i = gt; i < f.nodecnt_words; i += kAllThreads) f.node_cnt[i] = 0;
-    if (rank == 0) {
-        if (threadIdx.x < (int)(sizeof(WsHeader) / 4)) reinterpret_cast<unsigned*>(hdr)[threadIdx.x] = 0;
-        if (threadIdx.x < f.P.n) f.tab[threadIdx.x] = f.P.s[threadIdx.x];
-    }
-    for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(wh[warp])[s] = 0;
-
-    // ---- a1: load and validate.  Warp gw of the cluster owns entries [gw * lw, gw * lw + lw).
+    pdl_wait();
     const int gw = rank * kFrontWarps + warp;
-    const int ng = f.lw / 32;
-    unsigned key[kFrontGroups];
+    {
+        // ask for the indices now (into L2): the trip to memory overlaps the set-up below
+        int r = 0;
+#pragma unroll 1
+        for (int g = 0; g < ng; ++g) {
+            const int e = gw * f.lw + g * 32 + lane;
+            if (e < f.n_total) {
+                while (r + 1 < f.P.n && (long long)e >= f.P.s[r + 1].start) ++r;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const IT*>(f.P.s[r].indices) + ((long long)e - f.P.s[r].start)));
+            }
+        }
+    }
+    // The header (counters, flags) starts at zero; every CTA clears its own bitmap flag.  Only then may the
+    // row-reduction kernel start beside this one: it polls those flags.
+    if (rank == 0 && threadIdx.x < kHeaderWordsBeforeFlags) reinterpret_cast<unsigned*>(hdr)[threadIdx.x] = 0;
+    if (threadIdx.x == 0) hdr->bitmap_ready[rank] = 0;
+    for (int i = threadIdx.x; i < 2 * f.bitmap_words; i += kFrontThreads) reinterpret_cast<uint4*>(named)[i] = make_uint4(0u, 0u, 0u, 0u);
+    __threadfence();
+    __syncthreads();
+    pdl_trigger();
+    // ---- a1: load and validate.  Warp gw of the cluster owns entries [gw * lw, gw * lw + lw) of the input.
     {
         int r = 0;
-#pragma unroll
-        for (int g = 0; g < kFrontGroups; ++g) {
-            key[g] = kInvalidKey;
+#pragma unroll 1
+        for (int g = 0; g < ng; ++g) {
             const int e = gw * f.lw + g * 32 + lane;
-            if (g < ng && e < f.n_total) {
+            unsigned x = 0xFFFFFFFFu;
+            if (e < f.n_total) {
                 while (r + 1 < f.P.n && (long long)e >= f.P.s[r + 1].start) ++r;
                 const long long v = (long long)static_cast<const IT*>(f.P.s[r].indices)[(long long)e - f.P.s[r].start];
-                if (v >= 0 && v < f.vocab) key[g] = (unsigned)v;
+                if (v >= 0 && v < f.vocab) { x = ((unsigned)v << 16) | (unsigned)e; named[v] = 1; }   // everybody writes the same value
+            }
+            buf0[warp * f.lw + g * 32 + lane] = x;
+        }
+    }
+    // what else must start at zero or be in place before the tables are used
+    for (int i = gt; i < f.nodecnt_words; i += kAllThreads) f.node_cnt[i] = 0;
+    for (int i = gt; i < f.batch_max; i += kAllThreads) f.batches[i] = make_int2(0x7FFFFFFF, 0);
+    if (rank == 0 && threadIdx.x < f.P.n) f.tab[threadIdx.x] = f.P.s[threadIdx.x];
+    __syncthreads();
+    // ---- the named rows, 32 per word, as this CTA sees them: the other kernel ORs the eight copies
+    for (int w = threadIdx.x; w < f.bitmap_words; w += kFrontThreads) {
+        const uint4 lo = reinterpret_cast<const uint4*>(named)[2 * w], hi = reinterpret_cast<const uint4*>(named)[2 * w + 1];
+        const unsigned x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+        unsigned word = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) word |= (((x[i] & 0x01010101u) * 0x01020408u) >> 24) << (4 * i);   // four 0/1 bytes -> four bits
+        f.bitmap[w * kClusterCtas + rank] = word;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();                              // the words of every thread of this CTA, ordered by the barrier
+        *reinterpret_cast<volatile int*>(&hdr->bitmap_ready[rank]) = 1;
+    }
+    // ---- a4: two stable passes, low digit of the key first.  A pass takes this CTA's slice of `src` (warp w:
+    // entries [w * lw, w * lw + lw)) and sends every entry to the shared memory of the CTA that owns its
+    // position in the order by digit: base[part][digit] + wh[warp][digit] + its rank among its warp's
+    // entries with that digit.
+    int n_valid = 0;
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+        const unsigned* src = pass ? buf1 : buf0;
+        unsigned* dst = pass ? buf0 : buf1;
+        const int shift = 16 + 8 * pass;
+        const int bound = pass ? n_valid - rank * S : S;          // entries of the slice that exist
+        for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(dg.wh[warp])[s] = 0;
+        __syncwarp();
+#pragma unroll 1
+        for (int g = 0; g < ng; ++g) {
+            const int e = warp * f.lw + g * 32 + lane;
+            const unsigned x = e < bound ? src[e] : 0xFFFFFFFFu;
+            const bool valid = x != 0xFFFFFFFFu;
+            const unsigned d = (x >> shift) & 255u;
+            const unsigned m = match_digit_rolled(d, valid);
+            const int leader = valid ? __ffs(m) - 1 : lane;
+            unsigned pre = 0;
+            if (valid && lane == leader) { pre = dg.wh[warp][d]; dg.wh[warp][d] = (unsigned short)(pre + __popc(m)); }
+            pre = __shfl_sync(0xFFFFFFFFu, pre, leader);
+            __syncwarp();
+            rks[e] = (unsigned short)(pre + __popc(m & ((1u << lane) - 1u)));
+        }
+        __syncthreads();
+        {
+            // per digit: prefix over the warps of this CTA (in four parts), then over the CTAs of the cluster
+            const int d = threadIdx.x & 255, part = threadIdx.x >> 8;
+            unsigned run = 0;
+#pragma unroll 1
+            for (int w = part * 8; w < part * 8 + 8; ++w) { const unsigned t = dg.wh[w][d]; dg.wh[w][d] = (unsigned short)run; run += t; }
+            dg.part_tot[part][d] = (unsigned short)run;
+            __syncthreads();
+            unsigned pt[kFrontParts];
+#pragma unroll
+            for (int p = 0; p < kFrontParts; ++p) pt[p] = dg.part_tot[p][d];
+            if (part == 0) dg.cta_tot[d] = pt[0] + pt[1] + pt[2] + pt[3];
+            cluster.sync();                           // every CTA's per-digit totals are in place
+            if (threadIdx.x < 256) {
+                unsigned before = 0, all = 0;
+#pragma unroll
+                for (int c = 0; c < kClusterCtas; ++c) {
+                    const unsigned t = cluster.map_shared_rank(dg.cta_tot, c)[d];
+                    if (c < rank) before += t;
+                    all += t;
+                }
+                unsigned inc = all;                   // exclusive scan of the digit totals over the 256 digits
+#pragma unroll 1
+                for (int o = 1; o < 32; o <<= 1) { unsigned t = __shfl_up_sync(0xFFFFFFFFu, inc, o); if (lane >= o) inc += t; }
+                if (lane == 31) dg.warp_tot[warp] = inc;
+                asm volatile("bar.sync 1, 256;" ::: "memory");   // the eight warps that hold the digits
+                unsigned b = inc - all + before;
+                for (int w = 0; w < warp; ++w) b += dg.warp_tot[w];
+                if (threadIdx.x == 255) dg.total = b - before + all;
+#pragma unroll
+                for (int p = 0; p < kFrontParts; ++p) { dg.base[p][d] = b; b += pt[p]; }
+            }
+            __syncthreads();
+        }
+        if (pass == 0) n_valid = (int)dg.total;
+#pragma unroll 1
+        for (int g = 0; g < ng; ++g) {
+            const int e = warp * f.lw + g * 32 + lane;
+            const unsigned x = e < bound ? src[e] : 0xFFFFFFFFu;
+            if (x != 0xFFFFFFFFu) {
+                const unsigned d = (x >> shift) & 255u;
+                const unsigned q = dg.base[warp >> 3][d] + (unsigned)dg.wh[warp][d] + (unsigned)rks[e];
+                const unsigned owner = q / (unsigned)S;
+                cluster.map_shared_rank(dst, owner)[q - owner * (unsigned)S] = x;
+            }
+        }
+        cluster.sync();                               // the pass has landed everywhere
+    }
+    // ---- a2 + a3 + a5 + a6 in one walk over the sorted order (now in buf0).  Thread t of CTA c owns the ng
+    // consecutive entries from position c * S + t * ng.  First walk: what this thread's stretch knows (Seg);
+    // a scan over lanes, warps and CTAs gives every thread the stretch of everything before it; second
+    // walk: the tables.
+    const unsigned* sorted = buf0;
+    const int e0 = threadIdx.x * ng;
+    const int i0 = rank * S + e0;
+    const int n_mine = max(0, min(ng, n_valid - i0));
+    const int chunk_log = f.chunk_log;
+    unsigned k_first_prev = 0xFFFFFFFFu, k_last_next = 0xFFFFFFFFu;      // keys beside the stretch; no key looks like this
+    if (n_mine > 0) {
+        if (i0 > 0) k_first_prev = (e0 > 0 ? sorted[e0 - 1] : cluster.map_shared_rank(buf0, rank - 1)[S - 1]) >> 16;
+        if (i0 + ng < n_valid) k_last_next = (e0 + ng < S ? sorted[e0 + ng] : cluster.map_shared_rank(buf0, rank + 1)[0]) >> 16;
+    }
+    Seg mine = seg_identity();
+    {
+        unsigned kb = k_first_prev;
+#pragma unroll 1
+        for (int j = 0; j < n_mine; ++j) {
+            const unsigned k = sorted[e0 + j] >> 16;
+            const unsigned ka = j + 1 < n_mine ? sorted[e0 + j + 1] >> 16 : (j + 1 < ng ? 0xFFFFFFFFu : k_last_next);
+            if (kb != k) mine.lh = i0 + j;
+            if (ka != k) {
+                mine.nt += 1;
+                if (mine.lh >= 0) seg_add_row(mine, i0 + j - mine.lh + 1, chunk_log); else mine.bt = i0 + j;
+            }
+            kb = k;
+        }
+    }
+    // three levels of one scan: lanes of a warp, warps of the CTA, CTAs of the cluster.  Every warp runs
+    // every level (the barriers between them are for all); what the levels above the first compute is the
+    // same in every warp, and warp 0 keeps it.
+    Seg lane_excl = seg_identity();
+    {
+        Seg v = mine;
+#pragma unroll 1
+        for (int level = 0; level < 3; ++level) {
+            Seg excl;
+            const Seg incl = seg_warp_scan(v, excl, chunk_log);
+            if (level == 0) {
+                lane_excl = excl;
+                if (lane == 31) s_warp_seg[warp] = incl;
+                __syncthreads();
+                v = s_warp_seg[lane];
+            } else if (level == 1) {
+                if (warp == 0) { s_warp_pre[lane] = excl; if (lane == 31) s_cta_seg = incl; }
+                cluster.sync();                       // every CTA's stretch is in place
+                v = seg_identity();
+                if (warp == 0 && lane < kClusterCtas) v = *cluster.map_shared_rank(&s_cta_seg, lane);
+            } else {
+                const Seg before = seg_shfl(excl, rank), grand = seg_shfl(incl, kClusterCtas - 1);
+                if (warp == 0 && lane == 0) { s_before = before; s_grand = grand; }
+                __syncthreads();
             }
         }
     }
-    __syncwarp();
-    // ---- a4, pass 0: low digit; registers -> the shared memory of the CTA that owns the target position.
-    // rk[g] is the entry's rank among the warp's entries with the same digit; once the counters have
-    // become positions (cluster_bases) the target is wh[warp][digit] + rk[g].
-    unsigned short rk[kFrontGroups];
-#pragma unroll
-    for (int g = 0; g < kFrontGroups; ++g) {
-        rk[g] = 0;
-        if (g < ng) rk[g] = (unsigned short)rank_step(wh[warp], key[g] != kInvalidKey, key[g] & 255u, lane);
-    }
-    __syncthreads();
-    const int n_valid = (int)cluster_bases(cluster, wh, cta_tot, s_warp_tot, &s_total);
-#pragma unroll
-    for (int g = 0; g < kFrontGroups; ++g) {
-        if (g < ng && key[g] != kInvalidKey) {
-            const unsigned q = (unsigned)wh[warp][key[g] & 255u] + rk[g];
-            const unsigned owner = q / (unsigned)S;
-            cluster.map_shared_rank(packed, owner)[q - owner * (unsigned)S] =
-                (key[g] << 16) | (unsigned)(gw * f.lw + g * 32 + lane);
-        }
-    }
-    __syncthreads();                                  // every warp has read its positions
-    for (int s = lane; s < 128; s += 32) reinterpret_cast<unsigned*>(wh[warp])[s] = 0;
-    cluster.sync();                                   // all of pass 0 has landed
-    // ---- pass 1: high digit; this CTA's slice [rank * S, rank * S + S) -> perm (global) and skey (owner's shared memory)
-#pragma unroll
-    for (int g = 0; g < kFrontGroups; ++g) {
-        key[g] = kInvalidKey; rk[g] = 0;
-        const int e = warp * f.lw + g * 32 + lane;
-        if (g < ng) {
-            const bool valid = rank * S + e < n_valid;
-            const unsigned x = valid ? packed[e] : 0u;   // a packed entry (never 0xFFFFFFFF: positions stay below 65535)
-            rk[g] = (unsigned short)rank_step(wh[warp], valid, x >> 24, lane);
-            if (valid) key[g] = x;
-        }
-    }
-    __syncthreads();
-    cluster_bases(cluster, wh, cta_tot, s_warp_tot, &s_total);
-#pragma unroll
-    for (int g = 0; g < kFrontGroups; ++g) {
-        if (g < ng && key[g] != kInvalidKey) {
-            const unsigned x = key[g];
-            const unsigned q = (unsigned)wh[warp][x >> 24] + rk[g];
-            f.perm[q] = x & 0xFFFFu;
-            const unsigned owner = q / (unsigned)S;
-            cluster.map_shared_rank(skey, owner)[q - owner * (unsigned)S] = (unsigned short)(x >> 16);
-        }
-    }
-    cluster.sync();                                   // the sorted keys are in place
-    // ---- a2: run lengths.  The first entry of a run subtracts its position from count[key], the last
-    // adds its position + 1; count[] lives in shared memory, rows [c * Vs, c * Vs + Vs) in CTA c.
-    for (int e = threadIdx.x; e < S; e += kFrontThreads) {
-        const int i = rank * S + e;
-        if (i < n_valid) {
-            const unsigned k = skey[e];
-            unsigned prev = ~k, next = ~k;
-            if (i > 0) prev = e > 0 ? skey[e - 1] : cluster.map_shared_rank(skey, rank - 1)[S - 1];
-            if (i + 1 < n_valid) next = e + 1 < S ? skey[e + 1] : cluster.map_shared_rank(skey, rank + 1)[0];
-            const unsigned owner = k / (unsigned)Vs;
-            unsigned* c = cluster.map_shared_rank(cnt, owner) + (k - owner * (unsigned)Vs);
-            if (prev != k) atomicSub(c, (unsigned)i);
-            if (next != k) atomicAdd(c, (unsigned)i + 1u);
-        }
-    }
-    cluster.sync();                                   // count[] is complete
-    // ---- a3 + a5 + a6: scan of count[].  Thread t of CTA c owns rows c * Vs + t * rpt + [0, rpt).
-    IT* unique_rows = static_cast<IT*>(f.unique_rows);
-    const int chunk = f.chunk, B = f.batch_units, vocab = (int)f.vocab;
-    const int l0 = threadIdx.x * f.rpt;              // first owned row, local
-    const int e0 = rank * Vs + l0;                   // ... and global
-    int c[kFrontRpt];
-    Sum6 mine{};
-    int maxseg = 0;
-#pragma unroll
-    for (int q = 0; q < kFrontRpt; ++q) {
-        c[q] = q < f.rpt ? (int)cnt[l0 + q] : 0;
-        const int cc = c[q];
-        mine.v[0] += cc;
-        mine.v[1] += cc > 0;
-        if (q < f.rpt && e0 + q < vocab && !(f.compact && cc == 0)) mine.v[5] += row_units(cc, chunk);
-        if (cc > chunk) {
-            const int n = (cc + chunk - 1) / chunk;
-            mine.v[2] += 1; mine.v[3] += n; mine.v[4] += upper_nodes(n);
-        }
-        maxseg = max(maxseg, cc);
-    }
-    int prev_cost = 0;                               // units of the row before this thread's first one
-    if (e0 > 0 && e0 < f.vocab_pad) {
-        const unsigned pc = l0 > 0 ? cnt[l0 - 1] : cluster.map_shared_rank(cnt, rank - 1)[Vs - 1];
-        prev_cost = row_units((int)pc, chunk);
-    }
-    Sum6 inc = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-#pragma unroll
-        for (int q = 0; q < 6; ++q) {
-            int t = __shfl_up_sync(0xFFFFFFFFu, inc.v[q], o);
-            if (lane >= o) inc.v[q] += t;
-        }
-    }
-    for (int o = 16; o > 0; o >>= 1) maxseg = max(maxseg, __shfl_down_sync(0xFFFFFFFFu, maxseg, o));
-    if (lane == 31) {
-#pragma unroll
-        for (int q = 0; q < 6; ++q) s_scan[warp][q] = inc.v[q];
-    }
-    if (lane == 0) s_maxseg[warp] = maxseg;
-    __syncthreads();
-    if (warp == 0) {
-        // lane w holds warp w's sums: scan them, leave each warp's exclusive prefix and the CTA's sums
-        Sum6 ws, wi;
-#pragma unroll
-        for (int q = 0; q < 6; ++q) { ws.v[q] = s_scan[lane][q]; wi.v[q] = ws.v[q]; }
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-#pragma unroll
-            for (int q = 0; q < 6; ++q) {
-                int t = __shfl_up_sync(0xFFFFFFFFu, wi.v[q], o);
-                if (lane >= o) wi.v[q] += t;
+    {
+        IT* unique_rows = static_cast<IT*>(f.unique_rows);
+        Seg run = seg_combine(s_before, seg_combine(s_warp_pre[warp], lane_excl, chunk_log), chunk_log);
+        unsigned kb = k_first_prev;
+#pragma unroll 1
+        for (int j = 0; j < n_mine; ++j) {
+            const int i = i0 + j;
+            const unsigned x = sorted[e0 + j];
+            const unsigned k = x >> 16;
+            const unsigned ka = j + 1 < n_mine ? sorted[e0 + j + 1] >> 16 : (j + 1 < ng ? 0xFFFFFFFFu : k_last_next);
+            f.perm[i] = x & 0xFFFFu;
+            if (kb != k) run.lh = i;
+            if (ka != k) {
+                // the row k ends here: rank u among the named rows, entries [run.lh, i]
+                const int u = run.nt, cc = i - run.lh + 1;
+                f.urow[u] = (int)k;
+                f.uoff[u] = run.lh;
+                if (unique_rows) unique_rows[u] = (IT)k;
+                if (f.counts_out) f.counts_out[u] = cc;
+                if (cc > (1 << chunk_log))           // a6: a heavy row becomes chunk items and a combine tree
+                    f.heavy[run.nh] = HeavyInfo{(int)k, run.nc, run.nu, (int)(heavy_shape(cc, chunk_log) & 0xFFFFu), run.lh, cc, {0, 0}};
+                // light work items: the row belongs to the item its first unit falls into
+                atomicMin(&f.batches[run.un >> f.batch_log].x, u + 1);
+                atomicMax(&f.batches[run.un >> f.batch_log].y, u + 1);
+                run.nt += 1;
+                seg_add_row(run, cc, chunk_log);
             }
-        }
-#pragma unroll
-        for (int q = 0; q < 6; ++q) {
-            s_scan[lane][q] = wi.v[q] - ws.v[q];
-            if (lane == 31) cta_sum[q] = wi.v[q];
-        }
-        int m = s_maxseg[lane];
-        for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_down_sync(0xFFFFFFFFu, m, o));
-        if (lane == 0 && m > 0) atomicMax(&hdr->max_segment, m);
-    }
-    __syncthreads();
-    Sum6 run;
-#pragma unroll
-    for (int q = 0; q < 6; ++q) run.v[q] = inc.v[q] - mine.v[q] + s_scan[warp][q];
-    cluster.sync();                                   // every CTA's sums are in place
-    if (threadIdx.x < 6) {
-        int before = 0, all = 0;
-        for (int cc = 0; cc < kClusterCtas; ++cc) {
-            const int t = cluster.map_shared_rank(cta_sum, cc)[threadIdx.x];
-            if (cc < rank) before += t;
-            all += t;
-        }
-        s_before[threadIdx.x] = before;
-        s_grand[threadIdx.x] = all;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int q = 0; q < 6; ++q) run.v[q] += s_before[q];
-    if (e0 < f.vocab_pad) {
-        int rem = run.v[5] % B;                      // units before row e0, modulo the batch size
-        int b = run.v[5] / B;
-#pragma unroll
-        for (int q = 0; q < kFrontRpt; ++q) {
-            const int v = e0 + q;
-            if (q < f.rpt && v < f.vocab_pad) {
-                const int cc = c[q];
-                f.offsets[v] = run.v[0];
-                if (cc > 0) {
-                    if (unique_rows) unique_rows[run.v[1]] = (IT)v;
-                    if (f.counts_out) f.counts_out[run.v[1]] = cc;
-                    if (f.compact) {
-                        // the row batches list named rows only: row number and first entry by rank among them
-                        const int u = run.v[1];
-                        f.urow[u] = v;
-                        f.uoff[u] = run.v[0];
-                        const int cost = row_units(cc, chunk);
-                        atomicMin(&f.batches[b].x, u + 1);
-                        atomicMax(&f.batches[b].y, u + 1);
-                        rem += cost;
-                        if (rem >= B) { b += rem / B; rem %= B; }
-                    }
-                    run.v[1] += 1;
-                }
-                if (cc > chunk) {
-                    // a6: a heavy row becomes n chunk items and a combine tree
-                    const int n = (cc + chunk - 1) / chunk;
-                    f.heavy[run.v[2]] = HeavyInfo{v, run.v[3], run.v[4], n, run.v[0], cc, {0, 0}};
-                    run.v[2] += 1; run.v[3] += n; run.v[4] += upper_nodes(n);
-                }
-                run.v[0] += cc;
-                if (v < vocab && !f.compact) {
-                    // light work items: row v belongs to batch floor(units before v / batch size)
-                    const int cost = row_units(cc, chunk);
-                    if (v == 0 || prev_cost > rem) f.batches[b].x = v + 1;
-                    rem += cost;
-                    if (v == vocab - 1 || rem >= B) f.batches[b].y = v + 1;
-                    if (rem >= B) { b += rem / B; rem %= B; }
-                    prev_cost = cost;
-                }
-            }
+            kb = k;
         }
     }
-    cluster.sync();       // all tables and the header's max_segment are written; nobody reads a peer's shared memory after this
     if (rank == 0 && threadIdx.x == 0) {
-        f.offsets[f.vocab_pad] = s_grand[0];
-        if (f.compact) f.uoff[s_grand[1]] = s_grand[0];
-        hdr->n_valid = s_grand[0];
-        hdr->n_unique = s_grand[1];
-        hdr->n_heavy = s_grand[2];
-        hdr->n_chunks = s_grand[3];
-        hdr->n_upper = s_grand[4];
-        hdr->n_batches = s_grand[5] > 0 ? (s_grand[5] - 1) / B + 1 : 0;
+        const Seg g = s_grand;
+        f.uoff[g.nt] = n_valid;
+        hdr->n_valid = n_valid;
+        hdr->n_unique = g.nt;
+        hdr->n_heavy = g.nh;
+        hdr->n_chunks = g.nc;
+        hdr->n_upper = g.nu;
+        hdr->max_segment = g.mx;
+        hdr->n_batches = g.un > 0 ? ((g.un - 1) >> f.batch_log) + 1 : 0;
         const long long bad = (long long)f.n_total - n_valid;
         hdr->n_bad = (unsigned long long)bad;
         if (bad) raise_status(hdr, DST_ERR_INDEX_OUT_OF_RANGE);
         if (f.result) {
-            f.result->n_unique = s_grand[1];
+            f.result->n_unique = g.nt;
             f.result->n_out_of_range = bad;
-            f.result->max_segment = *reinterpret_cast<volatile int*>(&hdr->max_segment);
+            f.result->max_segment = g.mx;
         }
+    }
+    cluster.sync();       // every table and the header have landed; nobody reads a peer's shared memory after this
+    if (rank == 0 && threadIdx.x == 0) {
+        __threadfence();
+        *reinterpret_cast<volatile int*>(&hdr->tables_ready) = 1;
     }
 }
 
 cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStream_t stream) {
     FrontArgs f;
-    f.P = p.P; f.hdr = p.hdr; f.tab = p.tab; f.perm = p.perm; f.offsets = p.offsets; f.heavy = p.heavy;
-    f.unique_rows = p.unique_rows; f.counts_out = p.counts_out; f.result = p.result; f.batches = p.batches;
-    f.urow = p.urow; f.uoff = p.uoff; f.compact = p.compact;
-    f.node_cnt = p.node_cnt; f.vocab = p.vocab; f.n_total = p.n_total; f.vocab_pad = p.vocab_pad; f.chunk = p.chunk;
-    f.batch_units = p.batch_units; f.batch_max = p.batch_max; f.nodecnt_words = p.nodecnt_words;
-    f.copy_src = static_cast<const uint4*>(p.copy_src); f.copy_dst = static_cast<uint4*>(p.copy_dst);
-    f.copy_vecs = p.copy_bytes / 16;
-    f.copy_apply = p.copy_apply; f.copy_lr = p.copy_lr;
+    f.P = p.P; f.hdr = p.hdr; f.tab = p.tab; f.perm = p.perm; f.heavy = p.heavy;
+    f.unique_rows = p.unique_rows; f.counts_out = p.counts_out; f.result = p.result;
+    f.urow = p.urow; f.uoff = p.uoff;
+    f.node_cnt = p.node_cnt; f.vocab = p.vocab; f.n_total = p.n_total;
+    f.nodecnt_words = p.nodecnt_words; f.batches = p.batches; f.batch_max = p.batch_max;
+    f.batch_log = 0;
+    while ((2 << f.batch_log) <= p.batch_units) ++f.batch_log;            // items of 2^batch_log units: the power of two below batch_units
+    f.bitmap = p.bitmap; f.bitmap_words = p.bitmap_words;
+    f.chunk_log = 0;
+    while ((1 << f.chunk_log) < p.chunk) ++f.chunk_log;
+    if ((1 << f.chunk_log) != p.chunk) return cudaErrorInvalidValue;      // chunk lengths are powers of two
     const int per_warp = (p.n_total + kClusterCtas * kFrontWarps - 1) / (kClusterCtas * kFrontWarps);
     f.lw = (per_warp + 31) / 32 * 32;
     if (f.lw < 32) f.lw = 32;
-    f.rpt = (p.vocab_pad + kClusterCtas * kFrontThreads - 1) / (kClusterCtas * kFrontThreads);
-    if (f.rpt < 1) f.rpt = 1;
-    if (f.lw > 32 * kFrontGroups || f.rpt > kFrontRpt) return cudaErrorInvalidValue;
-    const size_t S = size_t(32) * f.lw, Vs = size_t(kFrontThreads) * f.rpt;
-    const size_t smem = S * 4 + Vs * 4 + S * 2;
-    cudaError_t e;
-    if (index_type == DST_I64)
-        e = cudaFuncSetAttribute(k_front_cluster<long long>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    else
-        e = cudaFuncSetAttribute(k_front_cluster<int>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (f.lw > 32 * kFrontGroups || (long long)p.bitmap_words * 32 < p.vocab) return cudaErrorInvalidValue;
+    const size_t S = size_t(32) * f.lw;
+    const size_t smem = S * 10 + size_t(32) * p.bitmap_words;   // S is a multiple of 1024: the byte map stays 16-byte aligned
+    static SmemOptIn opt_in[2];
+    const cudaError_t e = index_type == DST_I64 ? ensure_dynamic_smem(k_front_cluster<long long>, smem, opt_in[1])
+                                                : ensure_dynamic_smem(k_front_cluster<int>, smem, opt_in[0]);
     if (e != cudaSuccess) return e;
-    // Copy clusters: no more than can be resident beside the index cluster (a cluster needs eight free SMs of
-    // one GPC; clusters that start late would finish late, their share of the rows being fixed).
-    int copy_clusters = p.copy_clusters > 0 ? p.copy_clusters : 0;
-    if (copy_clusters > 0) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(kClusterCtas * (1 + copy_clusters)); cfg.blockDim = dim3(kFrontThreads); cfg.dynamicSmemBytes = smem;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = kClusterCtas; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        // the answer depends on the device and on the shared memory asked for: remembered per index type
-        static std::atomic<long long> cache[2];
-        const int which = index_type == DST_I64 ? 1 : 0;
-        int dev = 0;
-        (void)cudaGetDevice(&dev);
-        const long long key = ((long long)smem << 16) | ((long long)(dev & 0xFF) << 8);
-        const long long seen = cache[which].load();
-        int resident = 0;
-        if ((seen & ~0xFFLL) == key && (seen & 0xFF) != 0) {
-            resident = int(seen & 0xFF);
-        } else {
-            if (which) e = cudaOccupancyMaxActiveClusters(&resident, k_front_cluster<long long>, &cfg);
-            else e = cudaOccupancyMaxActiveClusters(&resident, k_front_cluster<int>, &cfg);
-            if (e != cudaSuccess) { (void)cudaGetLastError(); resident = 0; }
-            if (resident > 0) cache[which].store(key | (resident > 255 ? 255 : resident));
-        }
-        if (resident >= 2 && copy_clusters > resident - 1) copy_clusters = resident - 1;
-    }
-    const int grid = kClusterCtas * (1 + copy_clusters);
     if (index_type == DST_I64)
-        return launch_pdl(k_front_cluster<long long>, dim3(grid), dim3(kFrontThreads), smem, stream, f);
-    return launch_pdl(k_front_cluster<int>, dim3(grid), dim3(kFrontThreads), smem, stream, f);
+        return launch_pdl(k_front_cluster<long long>, dim3(kClusterCtas), dim3(kFrontThreads), smem, stream, f);
+    return launch_pdl(k_front_cluster<int>, dim3(kClusterCtas), dim3(kFrontThreads), smem, stream, f);
 }
 
 }  // namespace dst

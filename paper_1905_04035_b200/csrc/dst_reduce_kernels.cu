@@ -23,6 +23,14 @@
 //                 in index order, so the result does not depend on timing)
 //   row batches   consecutive output rows that are not heavy, about batch_units units' worth
 // Rows wider than one slot are processed as independent column blocks.
+//
+// Small inputs (the paper's per-worker batches against a vocabulary of tens of thousands of rows):
+// most output rows are named by nobody and only need their dense_in row, and the index work is a
+// latency chain.  There the kernel is launched beside the index cluster and starts with
+//   copy items    a few consecutive output rows, those a bitmap marks as named left out;
+// when the index cluster flags its tables complete the warps turn to the chunk items and row
+// batches (which then list named rows only), and finish whatever copy items are left.  The two
+// kinds of item write disjoint rows, so no order between them is needed.
 #include "dst_common.cuh"
 
 namespace dst {
@@ -159,11 +167,14 @@ enum : int {
 
 constexpr int kTabCache = 64;       // slices whose table is copied into shared memory
 constexpr int kHeavyCache = 1024;   // heavy rows whose first chunk id is copied into shared memory
+constexpr int kNamedWords = 65536 / 32;   // the overlapped path is for vocabularies of at most 65536 rows
 struct CtaTables {
     long long start[kTabCache];
     unsigned long long values[kTabCache];
     int chunk_base[kHeavyCache];
     int n_heavy;
+    int state;                     // overlapped path: 0 tables not loaded, 1 a warp is loading them, 2 loaded
+    unsigned named[kNamedWords];   // overlapped path: bit v set when some valid entry names row v
 };
 
 // A block of at most 32 units, one per lane.
@@ -176,7 +187,8 @@ struct UnitBlock {
 
 // APPLY: instead of writing the accumulated gradient, take the SGD step on the weight that `out` holds
 // (fp32 rows only): out <- out - lr * (dense_in + sum of value rows).
-template <typename VT, typename OT, int K, bool APPLY = false>
+// OVERLAP: the kernel runs beside the index cluster and starts with copy items (small inputs, see above).
+template <typename VT, typename OT, int K, bool APPLY = false, bool OVERLAP = false>
 struct WarpPipe {
     static constexpr int VC = 16 / sizeof(VT);     // columns per 16-byte group of a value row
     const MainArgs& a;
@@ -185,7 +197,7 @@ struct WarpPipe {
     const unsigned bars;      // shared address of this warp's first mbarrier (one per slot)
     char* const ring_ptr;     // generic address of the first slot
     volatile int* const abort_flag;
-    const CtaTables& tabs;    // this CTA's shared copies of the slice table and of the heavy rows' first chunk ids
+    CtaTables& tabs;          // this CTA's shared copies of the slice table and of the heavy rows' first chunk ids
     HeavyInfo cur_heavy;      // the heavy row of the chunk item being processed
     int islot;                // slot the next issued unit goes to
     int cslot;                // slot of the next unit to consume
@@ -193,7 +205,7 @@ struct WarpPipe {
     unsigned issued_mask;     // slots with a copy that may still be in flight
 
     __device__ WarpPipe(const MainArgs& args, unsigned ring_addr, unsigned bar_addr, char* ring_generic, volatile int* ab,
-                        const CtaTables& t)
+                        CtaTables& t)
         : a(args), lane(lane_id()), ring(ring_addr), bars(bar_addr), ring_ptr(ring_generic), abort_flag(ab), tabs(t), islot(0),
           cslot(0), cphase(0u), issued_mask(0u) {}
 
@@ -367,7 +379,7 @@ struct WarpPipe {
             constexpr bool kDenseInRing = sizeof(VT) == 4 && sizeof(OT) == 4;
             const float* dense_row = nullptr;
             if constexpr (kDenseInRing)
-                if (root && a.dense_in && !(APPLY && a.compact))   // a pre-filled weight already holds the dense part of the step
+                if (root && a.dense_in)
                     dense_row = static_cast<const float*>(a.dense_in) + (long long)hi.row * a.d + cb;
             if (!sum_children(acc, child_first + parent * kFanIn, n_children, cb, wcols, dense_row)) return false;
             if (root) {
@@ -517,8 +529,8 @@ struct WarpPipe {
         }
         const int o_next = __shfl_down_sync(0xFFFFFFFFu, o, 1);
         const int cnt = lane < nrows ? o_next - o : 0;
-        // APPLY, output not pre-filled: the dense row is one more unit to add, before the weight row closes the row
-        const bool dense_unit = APPLY && a.dense_in && !a.compact;
+        // APPLY: the dense row is one more unit to add, before the weight row closes the row
+        const bool dense_unit = APPLY && a.dense_in;
         const int nunits = (lane < nrows && cnt <= a.chunk) ? cnt + 1 + (dense_unit ? 1 : 0) : 0;   // heavy rows belong to the chunk items
         int incl = nunits;
 #pragma unroll
@@ -570,32 +582,169 @@ struct WarpPipe {
         return true;
     }
 
-    __device__ void run() {
-        const unsigned n_chunks = (unsigned)a.hdr->n_chunks;
-        const unsigned n_base = n_chunks + (unsigned)a.hdr->n_batches;
-        const unsigned n_items = n_base * (unsigned)a.ncb;
-        // The first item of a warp is its own number (no traffic on the shared counter while the whole
-        // grid starts up); later ones come from the counter, fetched one item ahead.
+    // A few consecutive output rows that only need their dense_in row (or zeros; APPLY: the dense part of
+    // the step): the rows of the item that the bitmap does not mark as named.
+    __device__ bool do_copy(unsigned item) {
+        const int groups = (a.vocab + a.copy_rows - 1) / a.copy_rows;
+        const int cblk = (int)(item / (unsigned)groups);
+        const int r0 = ((int)item - cblk * groups) * a.copy_rows;      // copy_rows divides 32: the rows share one bitmap word
+        const int n_valid = min(a.copy_rows, a.vocab - r0);
+        const unsigned span = n_valid >= 32 ? 0xFFFFFFFFu : ((1u << n_valid) - 1u);
+        const unsigned want = ~(tabs.named[r0 >> 5] >> (r0 & 31)) & span;
+        const int n = __popc(want);
+        if (n == 0) return true;
+        const long long cb = (long long)cblk * a.W;
+        const long long wcols = min((long long)a.W, a.d - cb);
+        const unsigned bytes = (unsigned)(wcols * (long long)sizeof(OT));
+        Acc<VC> acc[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) zero(acc[k]);
+        const int per_row = APPLY ? 2 : 1;
+        const int total = n * per_row;
+        for (int base = 0; base < total; base += 32) {
+            const int q = base + lane;
+            UnitBlock b{nullptr, 0u, 0, 0};
+            if (q < total) {
+                b.y = r0 + (int)__fns(want, 0u, q / per_row + 1);          // the (q / per_row + 1)-th row that is wanted
+                const long long at = (long long)b.y * a.d + cb;
+                if (APPLY && !(q & 1)) {
+                    b.src = static_cast<const OT*>(a.dense_in) + at; b.bytes = bytes; b.kind = kUnitAdd;
+                } else if (APPLY) {
+                    b.src = static_cast<const OT*>(a.out) + at; b.bytes = bytes; b.kind = kUnitFinal;
+                } else {
+                    b.kind = kUnitFinal | kUnitCopy;
+                    if (a.dense_in) { b.src = static_cast<const OT*>(a.dense_in) + at; b.bytes = bytes; }
+                }
+            }
+            if (!run_block(acc, b, min(32, total - base), cblk)) return false;
+        }
+        return true;
+    }
+
+    // Work items handed out through one counter.  While plenty of items are left the next one is
+    // claimed one item ahead, so its number is back from the counter before it is needed.  Near the
+    // end that would leave some warps with an extra item in hand while others have run dry: then a
+    // warp claims only when it is out of work.
+    struct Claim {
+        unsigned* counter;
+        unsigned n_items, base, item, pending;
+        bool lazy;
+    };
+    // static_first: the first item of a warp is its own number (no traffic on the counter while the
+    // whole grid starts up) and the counter hands out the numbers after those
+    __device__ __forceinline__ void claim_begin(Claim& c, unsigned* counter, unsigned n_items, bool static_first) {
         const unsigned n_warps = gridDim.x * (unsigned)kPipeWarps;
-        unsigned item = blockIdx.x * (unsigned)kPipeWarps + (unsigned)warp_id();
-        // While plenty of items are left, the next item is claimed one item ahead, so its number is
-        // back from the counter before it is needed.  Near the end that would leave some warps with
-        // an extra item in hand while others have run dry: then a warp claims only when it is out of work.
-        bool ok = true, lazy = n_items < 2u * n_warps;
-        unsigned pending = 0xFFFFFFFFu;
-        if (lane == 0 && item < n_items && !lazy) pending = n_warps + atomicAdd(&a.hdr->work_counter, 1u);
-        while (ok && item < n_items) {
-            const int cblk = (int)(item / n_base);
-            const unsigned base = item - (unsigned)cblk * n_base;
-            ok = base < n_chunks ? do_chunk((int)base, cblk) : do_rows((int)(base - n_chunks), cblk);
-            if (lazy) {
-                unsigned it = 0;
-                if (lane == 0) it = n_warps + atomicAdd(&a.hdr->work_counter, 1u);
-                item = __shfl_sync(0xFFFFFFFFu, it, 0);
-            } else {
-                item = __shfl_sync(0xFFFFFFFFu, pending, 0);
-                if (item < n_items && n_items - item < 2u * n_warps) lazy = true;
-                if (lane == 0 && item < n_items && !lazy) pending = n_warps + atomicAdd(&a.hdr->work_counter, 1u);
+        c.counter = counter; c.n_items = n_items; c.pending = 0xFFFFFFFFu;
+        c.lazy = n_items < 2u * n_warps;
+        if (static_first) {
+            c.base = n_warps;
+            c.item = blockIdx.x * (unsigned)kPipeWarps + (unsigned)warp_id();
+        } else {
+            c.base = 0;
+            unsigned it = 0;
+            if (lane == 0) it = atomicAdd(counter, 1u);
+            c.item = __shfl_sync(0xFFFFFFFFu, it, 0);
+        }
+        if (lane == 0 && c.item < n_items && !c.lazy) c.pending = c.base + atomicAdd(counter, 1u);
+    }
+    __device__ __forceinline__ void claim_next(Claim& c) {
+        const unsigned n_warps = gridDim.x * (unsigned)kPipeWarps;
+        if (c.lazy) {
+            unsigned it = 0;
+            if (lane == 0) it = c.base + atomicAdd(c.counter, 1u);
+            c.item = __shfl_sync(0xFFFFFFFFu, it, 0);
+        } else {
+            c.item = __shfl_sync(0xFFFFFFFFu, c.pending, 0);
+            if (c.item < c.n_items && c.n_items - c.item < 2u * n_warps) c.lazy = true;
+            if (lane == 0 && c.item < c.n_items && !c.lazy) c.pending = c.base + atomicAdd(c.counter, 1u);
+        }
+    }
+
+    // Overlapped path: the slice table and the heavy rows' first chunk ids come into shared memory once
+    // the index cluster has written them; the first warp of the CTA to get here loads them.
+    __device__ bool load_tables_once() {
+        int st = 0;
+        if (lane == 0) st = atomicCAS(&tabs.state, 0, 1);
+        st = __shfl_sync(0xFFFFFFFFu, st, 0);
+        if (st == 0) {
+            for (int r = lane; r < a.R; r += 32) {
+                tabs.start[r] = a.tab[r].start;
+                tabs.values[r] = reinterpret_cast<unsigned long long>(a.tab[r].values);
+            }
+            const int nh = a.hdr->n_heavy;
+            if (lane == 0) tabs.n_heavy = nh;
+            if (nh <= kHeavyCache)
+                for (int h = lane; h < nh; h += 32) tabs.chunk_base[h] = a.heavy[h].chunk_base;
+            __threadfence_block();
+            __syncwarp();
+            if (lane == 0) atomicExch(&tabs.state, 2);
+        } else if (st == 1) {
+            const long long start = clock64();
+            volatile int* state = &tabs.state;
+            while (*state != 2) {
+                if (*abort_flag || clock64() - start > kWaitCycles) { give_up(); return false; }
+            }
+            __threadfence_block();
+        }
+        __syncwarp();
+        return true;
+    }
+
+    __device__ void run() {
+        bool ok = true;
+        Claim copies{};
+        unsigned n_copy = 0;
+        if constexpr (OVERLAP) {
+            // Until the index cluster says its tables are complete: copy items.  The flag is asked for
+            // before an item and looked at after it, so the trip to memory costs nothing.
+            n_copy = (unsigned)((a.vocab + a.copy_rows - 1) / a.copy_rows) * (unsigned)a.ncb;
+            claim_begin(copies, &a.hdr->copy_counter, n_copy, true);
+            volatile int* ready_flag = &a.hdr->tables_ready;
+            bool ready = false;
+            while (ok && !ready) {
+                int f = 0;
+                bool waited = false;
+                if (lane == 0) f = *ready_flag;
+                if (copies.item < n_copy) {
+                    ok = do_copy(copies.item);
+                    claim_next(copies);
+                } else {
+                    // nothing left to copy: wait for the tables, within the limit
+                    waited = true;
+                    if (lane == 0) {
+                        const long long start = clock64();
+                        while (!f) {
+                            if (*abort_flag || clock64() - start > kWaitCycles) break;
+                            __nanosleep(200);
+                            f = *ready_flag;
+                        }
+                    }
+                }
+                ready = __shfl_sync(0xFFFFFFFFu, f, 0) != 0;
+                if (waited && !ready) { give_up(); ok = false; }   // the wait ran out
+            }
+            if (ok) {
+                __threadfence();        // the tables were written before the flag
+                ok = load_tables_once();
+            }
+        }
+        if (ok) {
+            const unsigned n_chunks = (unsigned)a.hdr->n_chunks;
+            const unsigned n_base = n_chunks + (unsigned)a.hdr->n_batches;
+            const unsigned n_items = n_base * (unsigned)a.ncb;
+            Claim c{};
+            claim_begin(c, &a.hdr->work_counter, n_items, !OVERLAP);
+            while (ok && c.item < n_items) {
+                const int cblk = (int)(c.item / n_base);
+                const unsigned base = c.item - (unsigned)cblk * n_base;
+                ok = base < n_chunks ? do_chunk((int)base, cblk) : do_rows((int)(base - n_chunks), cblk);
+                claim_next(c);
+            }
+        }
+        if constexpr (OVERLAP) {
+            while (ok && copies.item < n_copy) {      // the copy items that are left
+                ok = do_copy(copies.item);
+                claim_next(copies);
             }
         }
         if (!ok) {
@@ -610,7 +759,7 @@ struct WarpPipe {
     }
 };
 
-template <typename VT, typename OT, int K, bool APPLY = false>
+template <typename VT, typename OT, int K, bool APPLY = false, bool OVERLAP = false>
 __global__ void __launch_bounds__(kPipeThreads, sizeof(VT) == 2 ? 4 : 2)
 k_reduce_rows(const __grid_constant__ MainArgs a) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -625,26 +774,54 @@ k_reduce_rows(const __grid_constant__ MainArgs a) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     pdl_trigger();
-    pdl_wait();       // everything above overlaps with the tail of the kernel before
-    if (a.R <= kTabCache) {
-        for (int r = threadIdx.x; r < a.R; r += kPipeThreads) {
-            tabs.start[r] = a.tab[r].start;
-            tabs.values[r] = reinterpret_cast<unsigned long long>(a.tab[r].values);
+    if constexpr (!OVERLAP) {
+        pdl_wait();       // everything above overlaps with the tail of the kernel before
+        if (a.R <= kTabCache) {
+            for (int r = threadIdx.x; r < a.R; r += kPipeThreads) {
+                tabs.start[r] = a.tab[r].start;
+                tabs.values[r] = reinterpret_cast<unsigned long long>(a.tab[r].values);
+            }
         }
-    }
-    {
         const int nh = a.hdr->n_heavy;
         if (threadIdx.x == 0) tabs.n_heavy = nh;
         if (nh <= kHeavyCache)
             for (int h = threadIdx.x; h < nh; h += kPipeThreads) tabs.chunk_base[h] = a.heavy[h].chunk_base;
+    } else {
+        // Running beside the index cluster (which cleared the header before it let this kernel start, and
+        // which waited for everything earlier in the stream): first the bitmap of named rows, one copy per
+        // CTA of that cluster, each flagged when written.
+        if (threadIdx.x == 0) tabs.state = 0;
+        if (warp == 0) {
+            volatile const int* flags = a.hdr->bitmap_ready;
+            const long long start = clock64();
+            while (true) {
+                const int v = lane_id() < kClusterCtas ? flags[lane_id()] : 1;
+                if (__all_sync(0xFFFFFFFFu, v != 0)) break;
+                if (clock64() - start > kWaitCycles) {
+                    if (lane_id() == 0) { raise_status(a.hdr, DST_ERR_TIMEOUT); s_abort = 1; }
+                    break;
+                }
+                __nanosleep(100);
+            }
+        }
+        __syncthreads();
+        if (!s_abort) {
+            __threadfence();
+            for (int w = threadIdx.x; w < a.bitmap_words; w += kPipeThreads) {
+                const uint4 lo = __ldcg(reinterpret_cast<const uint4*>(a.bitmap) + 2 * w);
+                const uint4 hi = __ldcg(reinterpret_cast<const uint4*>(a.bitmap) + 2 * w + 1);
+                tabs.named[w] = lo.x | lo.y | lo.z | lo.w | hi.x | hi.y | hi.z | hi.w;
+            }
+        }
     }
     __syncthreads();
     {
         char* my_ring = slot_base + (size_t)warp * (size_t)a.n_slots * (size_t)a.slot_bytes;
-        WarpPipe<VT, OT, K, APPLY> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort, tabs);
+        WarpPipe<VT, OT, K, APPLY, OVERLAP> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort, tabs);
         // after a failed wait in an earlier kernel the tables are not to be trusted: touch nothing
-        if (*reinterpret_cast<volatile int*>(&a.hdr->status) != DST_ERR_TIMEOUT) pipe.run();
+        if (OVERLAP ? !s_abort : *reinterpret_cast<volatile int*>(&a.hdr->status) != DST_ERR_TIMEOUT) pipe.run();
     }
+    if constexpr (OVERLAP) pdl_wait();   // nothing later in the stream may start before the index cluster has retired too
     __syncthreads();
     // the last CTA to finish reports the status word (it may have been raised by this kernel)
     if (threadIdx.x == 0 && a.result) {
@@ -686,20 +863,34 @@ k_reduce_rows_scalar(const MainArgs a) {
 // index lookup, a node of a combine tree), which is what a short call is made of.
 constexpr long long kInFlightBytes = 14ll << 20;
 
-template <typename VT, typename OT, int K, bool APPLY>
-static cudaError_t launch_pipe(MainArgs a, int sm_count, cudaStream_t stream) {
+template <typename VT, typename OT, int K, bool APPLY, bool OVERLAP>
+static cudaError_t launch_pipe_as(MainArgs a, int sm_count, cudaStream_t stream) {
     auto smem_for = [&](int slots) { return size_t(kPipeHeaderReserve) + size_t(kPipeWarps) * size_t(slots) * size_t(a.slot_bytes); };
-    cudaError_t e = cudaFuncSetAttribute(k_reduce_rows<VT, OT, K, APPLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_for(kPipeSlots));
+    // the shared-memory opt-in and the occupancy answer are asked of the runtime once per device and variant
+    static SmemOptIn opt_in;
+    static std::atomic<int> resident_on[64];
+    cudaError_t e = ensure_dynamic_smem(k_reduce_rows<VT, OT, K, APPLY, OVERLAP>, smem_for(kPipeSlots), opt_in);
     if (e != cudaSuccess) return e;
-    int resident = 0;                                    // CTAs of this variant an SM holds with full rings
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, k_reduce_rows<VT, OT, K, APPLY>, kPipeThreads, smem_for(kPipeSlots));
-    if (e != cudaSuccess) return e;
-    if (resident < 1) return cudaErrorLaunchOutOfResources;
+    int dev = -1, resident = 0;                          // CTAs of this variant an SM holds with full rings
+    const bool cached = cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64;
+    if (cached) resident = resident_on[dev].load();
+    if (resident < 1) {
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, k_reduce_rows<VT, OT, K, APPLY, OVERLAP>, kPipeThreads, smem_for(kPipeSlots));
+        if (e != cudaSuccess) return e;
+        if (resident < 1) return cudaErrorLaunchOutOfResources;
+        if (cached) resident_on[dev].store(resident);
+    }
     const int grid = sm_count * resident;
     const long long per_slot = (long long)grid * kPipeWarps * a.slot_bytes;
     long long slots = kInFlightBytes / per_slot;
     a.n_slots = (int)(slots < 2 ? 2 : (slots > kPipeSlots ? kPipeSlots : slots));
-    return launch_pdl(k_reduce_rows<VT, OT, K, APPLY>, dim3(grid), dim3(kPipeThreads), smem_for(a.n_slots), stream, a);
+    return launch_pdl(k_reduce_rows<VT, OT, K, APPLY, OVERLAP>, dim3(grid), dim3(kPipeThreads), smem_for(a.n_slots), stream, a);
+}
+
+template <typename VT, typename OT, int K, bool APPLY>
+static cudaError_t launch_pipe(const MainArgs& a, int sm_count, cudaStream_t stream) {
+    return a.overlap ? launch_pipe_as<VT, OT, K, APPLY, true>(a, sm_count, stream)
+                     : launch_pipe_as<VT, OT, K, APPLY, false>(a, sm_count, stream);
 }
 
 template <typename VT, typename OT, bool APPLY = false>
@@ -714,6 +905,11 @@ static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaSt
     }
     const PipeShape ps = pipe_shape((int)sizeof(VT), (int)sizeof(OT), a.d);
     a.W = ps.W; a.ncb = ps.ncb; a.slot_bytes = ps.slot_bytes; a.n_slots = ps.n_slots;
+    {
+        // a copy item: about 32 KB worth of consecutive rows, 8 to 32 of them
+        const long long row_bytes = (long long)ps.W * (long long)sizeof(OT);
+        a.copy_rows = row_bytes * 32 <= 32768 ? 32 : (row_bytes * 16 <= 32768 ? 16 : 8);
+    }
     constexpr int kMaxK = sizeof(VT) == 4 ? 8 : 4;
     if (ps.K == 1) return launch_pipe<VT, OT, 1, APPLY>(a, sm_count, stream);
     if (ps.K == 2) return launch_pipe<VT, OT, 2, APPLY>(a, sm_count, stream);
