@@ -99,12 +99,11 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         fp.hdr = hdr; fp.tab = tab; fp.perm = pos[0]; fp.heavy = heavy;
         fp.unique_rows = unique_rows; fp.counts_out = counts; fp.result = result;
         fp.node_cnt = nodecnt; fp.vocab = vocab; fp.n_total = int(n_total);
-        fp.chunk = L.chunk; fp.batch_units = L.batch_units; fp.batches = batches; fp.batch_max = int(L.batch_max);
+        fp.chunk = L.chunk; fp.batch_units = L.batch_units; fp.bfirst = reinterpret_cast<int*>(batches);
         fp.nodecnt_words = int((L.off_batches - L.off_nodecnt) / 4);
         compact = true;
         overlap = apply ? dense_in != nullptr : out != dense_in;
-        fp.urow = reinterpret_cast<int*>(ws + L.off_urow);
-        fp.uoff = reinterpret_cast<int*>(ws + L.off_uoff);
+        fp.urec = reinterpret_cast<unsigned*>(ws + L.off_urow);
         fp.bitmap = reinterpret_cast<unsigned*>(ws + L.off_bitmap);
         fp.bitmap_words = L.bitmap_words;
         if (launch_front_cluster(opts->index_type, fp, stream) != cudaSuccess) return DST_ERR_CUDA;
@@ -163,10 +162,9 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     a.overlap = overlap ? 1 : 0;
     a.bitmap = reinterpret_cast<const unsigned*>(ws + L.off_bitmap);
     a.bitmap_words = L.bitmap_words;
-    a.copy_rows = 8;     // set by the launcher
+    a.copy_rows = 8; a.copy_slots = 0;     // set by the launcher
     a.apply = apply ? 1 : 0; a.lr = lr;
-    a.urow = reinterpret_cast<const int*>(ws + L.off_urow);
-    a.uoff = reinterpret_cast<const int*>(ws + L.off_uoff);
+    a.urec = reinterpret_cast<const unsigned*>(ws + L.off_urow);
     if (t_ev_before && cudaEventRecord(t_ev_before, stream) != cudaSuccess) return DST_ERR_CUDA;
     if (launch_reduce_rows(a, opts->value_type, opts->out_type, vector_ok, sm_count(), stream) != cudaSuccess)
         return DST_ERR_CUDA;

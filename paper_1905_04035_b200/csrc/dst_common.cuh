@@ -116,9 +116,10 @@ struct MainArgs {
     const unsigned* perm;
     const SliceEntry* tab;
     const HeavyInfo* heavy;
-    const int2* batches;   // per row batch: first row + 1, last row + 1 (0: empty batch); `compact`: ranks among the named rows
-    const int* urow;       // compact: the named rows, ascending
-    const int* uoff;       // compact: first entry of each named row in perm[], then the number of entries
+    const int2* batches;   // per row batch: first row + 1, last row + 1 (0: empty batch).  `compact`: an int per batch
+                           // instead, the rank of its first named row, and one more int, the number of named rows
+    const unsigned* urec;  // compact: the named rows by rank: row << 16 | first entry in perm[]; then the number of entries
+                           // (and perm[] holds 16-bit positions)
     unsigned* node_cnt;
     float* partials;
     const void* dense_in;
@@ -143,6 +144,7 @@ struct MainArgs {
     // then it takes the named rows, then whatever copy items are left.
     int overlap;
     int copy_rows;              // rows per copy item: 8, 16 or 32 (a divisor of 32)
+    int copy_slots;             // ring slots in use while copying (n_slots while reducing)
     const unsigned* bitmap;     // kClusterCtas interleaved copies, see Layout::off_bitmap
     int bitmap_words;
 };
@@ -249,11 +251,10 @@ struct FrontParams {
     int* counts_out;
     dst_result_t* result;
     unsigned* node_cnt;
-    int2* batches;
+    int* bfirst;               // light work items: rank of the first named row of each, then the number of named rows
     long long vocab;
-    int n_total, chunk, batch_units, batch_max, nodecnt_words;
-    int* urow;                 // the named rows, ascending
-    int* uoff;                 // first entry of each named row in perm[], then the number of entries
+    int n_total, chunk, batch_units, nodecnt_words;
+    unsigned* urec;            // the named rows, ascending: row << 16 | first entry in perm[]; then the number of entries
     unsigned* bitmap;          // named-row bitmap, written early for the row-reduction kernel running beside this one
     int bitmap_words;
 };

@@ -38,18 +38,17 @@ struct FrontArgs {
     HistParams P;              // the slices
     WsHeader* hdr;
     SliceEntry* tab;
-    unsigned* perm;
+    unsigned short* perm;      // input positions in sorted order, 16 bits each
     HeavyInfo* heavy;
     void* unique_rows;
     int* counts_out;
     dst_result_t* result;
-    int* urow;
-    int* uoff;
+    unsigned* urec;            // per named row, by rank: row << 16 | first entry in perm; one more word holds the number of entries
     unsigned* node_cnt;
-    int2* batches;             // light work items: ranks (+ 1) of the first and last named row that start in each
+    int* bfirst;               // light work items: rank of the first named row of each; one more entry holds the number of named rows
     unsigned* bitmap;          // [bitmap_words][kClusterCtas]: this CTA's copy of the named-row bitmap at [w * 8 + rank]
     long long vocab;
-    int n_total, chunk_log, batch_log, batch_max, nodecnt_words, bitmap_words;
+    int n_total, chunk_log, batch_log, nodecnt_words, bitmap_words;
     int lw;                    // entries per warp (multiple of 32); a CTA's slice of the sorted order holds 32 * lw
 };
 
@@ -66,7 +65,7 @@ constexpr int kFrontParts = 4;        // the warps of a CTA in four parts of eig
 // Lanes of the warp whose 8-bit digit equals this lane's, among the lanes with `valid` set.
 __device__ __forceinline__ unsigned match_digit_rolled(unsigned dg, bool valid) {
     unsigned m = __ballot_sync(0xFFFFFFFFu, valid);
-#pragma unroll 1
+#pragma unroll           // the one loop of this file that is unrolled: the ranking is bound by the instructions issued
     for (int b = 0; b < 8; ++b) {
         const bool bit = (dg >> b) & 1u;
         const unsigned bal = __ballot_sync(0xFFFFFFFFu, bit);
@@ -216,10 +215,6 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
             buf0[warp * f.lw + g * 32 + lane] = x;
         }
     }
-    // what else must start at zero or be in place before the tables are used
-    for (int i = gt; i < f.nodecnt_words; i += kAllThreads) f.node_cnt[i] = 0;
-    for (int i = gt; i < f.batch_max; i += kAllThreads) f.batches[i] = make_int2(0x7FFFFFFF, 0);
-    if (rank == 0 && threadIdx.x < f.P.n) f.tab[threadIdx.x] = f.P.s[threadIdx.x];
     __syncthreads();
     // ---- the named rows, 32 per word, as this CTA sees them: the other kernel ORs the eight copies
     for (int w = threadIdx.x; w < f.bitmap_words; w += kFrontThreads) {
@@ -235,6 +230,9 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
         __threadfence();                              // the words of every thread of this CTA, ordered by the barrier
         *reinterpret_cast<volatile int*>(&hdr->bitmap_ready[rank]) = 1;
     }
+    // what else must start at zero or be in place before the tables are used
+    for (int i = gt; i < f.nodecnt_words; i += kAllThreads) f.node_cnt[i] = 0;
+    if (rank == 0 && threadIdx.x < f.P.n) f.tab[threadIdx.x] = f.P.s[threadIdx.x];
     // ---- a4: two stable passes, low digit of the key first.  A pass takes this CTA's slice of `src` (warp w:
     // entries [w * lw, w * lw + lw)) and sends every entry to the shared memory of the CTA that owns its
     // position in the order by digit: base[part][digit] + wh[warp][digit] + its rank among its warp's
@@ -340,29 +338,30 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
             kb = k;
         }
     }
-    // three levels of one scan: lanes of a warp, warps of the CTA, CTAs of the cluster.  Every warp runs
-    // every level (the barriers between them are for all); what the levels above the first compute is the
-    // same in every warp, and warp 0 keeps it.
+    // three levels of one scan: lanes of a warp (every warp), then warps of the CTA and CTAs of the cluster
+    // (warp 0; the barriers between the levels are for all)
     Seg lane_excl = seg_identity();
     {
         Seg v = mine;
 #pragma unroll 1
         for (int level = 0; level < 3; ++level) {
-            Seg excl;
-            const Seg incl = seg_warp_scan(v, excl, chunk_log);
+            Seg excl = seg_identity(), incl = seg_identity();
+            if (level == 0 || warp == 0) incl = seg_warp_scan(v, excl, chunk_log);
             if (level == 0) {
                 lane_excl = excl;
                 if (lane == 31) s_warp_seg[warp] = incl;
                 __syncthreads();
-                v = s_warp_seg[lane];
+                if (warp == 0) v = s_warp_seg[lane];
             } else if (level == 1) {
                 if (warp == 0) { s_warp_pre[lane] = excl; if (lane == 31) s_cta_seg = incl; }
                 cluster.sync();                       // every CTA's stretch is in place
                 v = seg_identity();
                 if (warp == 0 && lane < kClusterCtas) v = *cluster.map_shared_rank(&s_cta_seg, lane);
             } else {
-                const Seg before = seg_shfl(excl, rank), grand = seg_shfl(incl, kClusterCtas - 1);
-                if (warp == 0 && lane == 0) { s_before = before; s_grand = grand; }
+                if (warp == 0) {
+                    const Seg before = seg_shfl(excl, rank), grand = seg_shfl(incl, kClusterCtas - 1);
+                    if (lane == 0) { s_before = before; s_grand = grand; }
+                }
                 __syncthreads();
             }
         }
@@ -370,27 +369,41 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
     {
         IT* unique_rows = static_cast<IT*>(f.unique_rows);
         Seg run = seg_combine(s_before, seg_combine(s_warp_pre[warp], lane_excl, chunk_log), chunk_log);
+        const int B = 1 << f.batch_log;
         unsigned kb = k_first_prev;
+        unsigned long long pw = 0;                       // up to four 16-bit positions on their way to perm
 #pragma unroll 1
         for (int j = 0; j < n_mine; ++j) {
             const int i = i0 + j;
             const unsigned x = sorted[e0 + j];
             const unsigned k = x >> 16;
             const unsigned ka = j + 1 < n_mine ? sorted[e0 + j + 1] >> 16 : (j + 1 < ng ? 0xFFFFFFFFu : k_last_next);
-            f.perm[i] = x & 0xFFFFu;
+            pw |= (unsigned long long)(x & 0xFFFFu) << (16 * (j & 3));
+            if ((j & 3) == 3 || j == n_mine - 1) {
+                // i0 is a multiple of ng: with ng a multiple of four this is one aligned 8-byte store
+                if ((ng & 3) == 0) {
+                    *reinterpret_cast<unsigned long long*>(f.perm + (i & ~3)) = pw;
+                } else {
+                    for (int q = 0; q <= (j & 3); ++q) f.perm[(i0 + (j & ~3)) + q] = (unsigned short)(pw >> (16 * q));
+                }
+                pw = 0;
+            }
             if (kb != k) run.lh = i;
             if (ka != k) {
                 // the row k ends here: rank u among the named rows, entries [run.lh, i]
                 const int u = run.nt, cc = i - run.lh + 1;
-                f.urow[u] = (int)k;
-                f.uoff[u] = run.lh;
+                f.urec[u] = (k << 16) | (unsigned)run.lh;
                 if (unique_rows) unique_rows[u] = (IT)k;
                 if (f.counts_out) f.counts_out[u] = cc;
                 if (cc > (1 << chunk_log))           // a6: a heavy row becomes chunk items and a combine tree
                     f.heavy[run.nh] = HeavyInfo{(int)k, run.nc, run.nu, (int)(heavy_shape(cc, chunk_log) & 0xFFFFu), run.lh, cc, {0, 0}};
-                // light work items: the row belongs to the item its first unit falls into
-                atomicMin(&f.batches[run.un >> f.batch_log].x, u + 1);
-                atomicMax(&f.batches[run.un >> f.batch_log].y, u + 1);
+                // Light work items: a row belongs to the item its first unit falls into, item b = units
+                // [b * B, b * B + B).  The row whose units reach or cross the start of an item names the
+                // next row as that item's first (an item no row starts in gets the same first row as the
+                // item after it, and is empty).
+                const int p0 = run.un, p1 = run.un + row_units(cc, 1 << chunk_log);
+                if (u == 0) f.bfirst[0] = 0;
+                for (int b = (p0 >> f.batch_log) + 1; b * B <= p1; ++b) f.bfirst[b] = u + 1;
                 run.nt += 1;
                 seg_add_row(run, cc, chunk_log);
             }
@@ -399,7 +412,8 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
     }
     if (rank == 0 && threadIdx.x == 0) {
         const Seg g = s_grand;
-        f.uoff[g.nt] = n_valid;
+        f.urec[g.nt] = (unsigned)n_valid;
+        f.bfirst[g.un > 0 ? ((g.un - 1) >> f.batch_log) + 1 : 0] = g.nt;
         hdr->n_valid = n_valid;
         hdr->n_unique = g.nt;
         hdr->n_heavy = g.nh;
@@ -425,11 +439,11 @@ k_front_cluster(const __grid_constant__ FrontArgs f) {
 
 cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStream_t stream) {
     FrontArgs f;
-    f.P = p.P; f.hdr = p.hdr; f.tab = p.tab; f.perm = p.perm; f.heavy = p.heavy;
+    f.P = p.P; f.hdr = p.hdr; f.tab = p.tab; f.perm = reinterpret_cast<unsigned short*>(p.perm); f.heavy = p.heavy;
     f.unique_rows = p.unique_rows; f.counts_out = p.counts_out; f.result = p.result;
-    f.urow = p.urow; f.uoff = p.uoff;
+    f.urec = p.urec; f.bfirst = p.bfirst;
     f.node_cnt = p.node_cnt; f.vocab = p.vocab; f.n_total = p.n_total;
-    f.nodecnt_words = p.nodecnt_words; f.batches = p.batches; f.batch_max = p.batch_max;
+    f.nodecnt_words = p.nodecnt_words;
     f.batch_log = 0;
     while ((2 << f.batch_log) <= p.batch_units) ++f.batch_log;            // items of 2^batch_log units: the power of two below batch_units
     f.bitmap = p.bitmap; f.bitmap_words = p.bitmap_words;

@@ -162,7 +162,8 @@ enum : int {
     kUnitAdd = 1,        // slot holds a value row: add it
     kUnitFinal = 2,      // finish output row y (slot holds its dense_in row unless there is no dense_in)
     kUnitCopy = 4,       // with kUnitFinal: nobody names the row, out = dense_in bit for bit
-    kUnitChunkEnd = 8    // last entry of chunk y: store the partial row, climb the tree
+    kUnitChunkEnd = 8,   // last entry of chunk y: store the partial row, climb the tree
+    kUnitPoll = 16       // (copy items) ask now whether the index cluster has finished; the answer is looked at after the item
 };
 
 constexpr int kTabCache = 64;       // slices whose table is copied into shared memory
@@ -203,11 +204,13 @@ struct WarpPipe {
     int cslot;                // slot of the next unit to consume
     unsigned cphase;          // bit s: parity to wait for on slot s
     unsigned issued_mask;     // slots with a copy that may still be in flight
+    int polled;               // lane 0: tables_ready as last asked for (kUnitPoll)
+    int ns;                   // slots of the ring in use (<= a.n_slots, the slots there are); changed only when the ring is empty
 
     __device__ WarpPipe(const MainArgs& args, unsigned ring_addr, unsigned bar_addr, char* ring_generic, volatile int* ab,
                         CtaTables& t)
         : a(args), lane(lane_id()), ring(ring_addr), bars(bar_addr), ring_ptr(ring_generic), abort_flag(ab), tabs(t), islot(0),
-          cslot(0), cphase(0u), issued_mask(0u) {}
+          cslot(0), cphase(0u), issued_mask(0u), polled(0), ns(args.n_slots) {}
 
     __device__ __forceinline__ int col(int k) const { return (k * 32 + lane) * VC; }
 
@@ -223,7 +226,7 @@ struct WarpPipe {
             }
         }
         issued_mask |= 1u << islot;
-        islot = islot + 1 == a.n_slots ? 0 : islot + 1;
+        islot = islot + 1 == ns ? 0 : islot + 1;
     }
 
     // position in the virtual concatenation -> address of that value row (slice table in shared memory)
@@ -247,7 +250,7 @@ struct WarpPipe {
             bulk_load(ring + (unsigned)islot * (unsigned)a.slot_bytes, src, bytes, bar);
         }
         issued_mask |= 1u << islot;
-        islot = islot + 1 == a.n_slots ? 0 : islot + 1;
+        islot = islot + 1 == ns ? 0 : islot + 1;
     }
 
     // acc = child[0] + child[1] + ... in index order.  fp32 value rows: a slot of the ring holds one
@@ -267,7 +270,7 @@ struct WarpPipe {
             for (int k = 0; k < K; ++k) zero(acc[k]);
             const unsigned bytes = (unsigned)wcols * 4u;
             int issued = 0;
-            for (; issued < n && issued < a.n_slots; ++issued) issue_plain(source(issued), bytes);
+            for (; issued < n && issued < ns; ++issued) issue_plain(source(issued), bytes);
             for (int c = 0; c < n; ++c) {
                 if (!mbar_wait(bars + 8u * (unsigned)cslot, (cphase >> cslot) & 1u, abort_flag)) { give_up(); return false; }
                 cphase ^= 1u << cslot;
@@ -283,7 +286,7 @@ struct WarpPipe {
 #pragma unroll
                 for (int k = 0; k < K; ++k) add(acc[k], v[k]);
                 __syncwarp();
-                cslot = cslot + 1 == a.n_slots ? 0 : cslot + 1;
+                cslot = cslot + 1 == ns ? 0 : cslot + 1;
                 if (issued < n) { issue_plain(source(issued), bytes); ++issued; }
             }
             return true;
@@ -437,11 +440,13 @@ struct WarpPipe {
         const long long cb = (long long)cblk * a.W;
         const int wcols = (int)min((long long)a.W, a.d - cb);
         OT* const out = static_cast<OT*>(a.out);
-        const int ahead = min(n, a.n_slots);
+        const int ahead = min(n, ns);
         for (int j = 0; j < ahead; ++j) issue(b, j);
         for (int j = 0; j < n; ++j) {
             const int kind = __shfl_sync(0xFFFFFFFFu, b.kind, j);
             const int y = __shfl_sync(0xFFFFFFFFu, b.y, j);
+            if constexpr (OVERLAP)
+                if ((kind & kUnitPoll) && lane == 0) polled = *reinterpret_cast<volatile int*>(&a.hdr->tables_ready);
             if (!mbar_wait(bars + 8u * (unsigned)cslot, (cphase >> cslot) & 1u, abort_flag)) { give_up(); return false; }
             cphase ^= 1u << cslot;
             issued_mask &= ~(1u << cslot);
@@ -481,8 +486,8 @@ struct WarpPipe {
                 }
             }
             __syncwarp();                                 // every lane has read the slot
-            cslot = cslot + 1 == a.n_slots ? 0 : cslot + 1;
-            if (j + a.n_slots < n) issue(b, j + a.n_slots);   // refill it
+            cslot = cslot + 1 == ns ? 0 : cslot + 1;
+            if (j + ns < n) issue(b, j + ns);   // refill it
             if (kind & kUnitChunkEnd) {
                 if (!finish_chunk(acc, y, cblk)) return false;
 #pragma unroll
@@ -503,7 +508,7 @@ struct WarpPipe {
             const int q = base + lane;
             UnitBlock b{nullptr, 0u, 0, cid};
             if (q < cd.len) {
-                const unsigned p = a.perm[cd.begin + q];
+                const unsigned p = a.compact ? reinterpret_cast<const unsigned short*>(a.perm)[cd.begin + q] : a.perm[cd.begin + q];
                 if (p < (unsigned)a.n_total) { b.src = row_address(p) + cb; b.bytes = bytes; b.kind = kUnitAdd; }
                 if (q == cd.len - 1) b.kind |= kUnitChunkEnd;
             }
@@ -514,16 +519,26 @@ struct WarpPipe {
 
     // A batch of consecutive output rows: their entries and their closing units, flattened
     __device__ bool do_rows(int batch, int cblk) {
-        const int2 bt = a.batches[batch];
-        if (bt.y == 0) return true;                       // no row starts in this batch
-        const int v0 = bt.x - 1;                          // first row (compact: its rank among the named rows)
-        const int nrows = min(bt.y - bt.x + 1, 31);
+        int v0, nrows;                                    // first row (compact: its rank among the named rows), rows
+        if (a.compact) {
+            const int* first = reinterpret_cast<const int*>(a.batches);
+            v0 = first[batch];
+            nrows = min(first[batch + 1] - v0, 31);
+            if (nrows <= 0) return true;                  // no row starts in this batch
+        } else {
+            const int2 bt = a.batches[batch];
+            if (bt.y == 0) return true;
+            v0 = bt.x - 1;
+            nrows = min(bt.y - bt.x + 1, 31);
+        }
         const long long cb = (long long)cblk * a.W;
         const long long wcols = min((long long)a.W, a.d - cb);
         int o = 0, row = v0 + lane;
         if (a.compact) {
-            if (lane <= nrows) o = a.uoff[v0 + lane];
-            if (lane < nrows) row = a.urow[v0 + lane];
+            if (lane <= nrows) {
+                const unsigned rec = a.urec[v0 + lane];
+                o = (int)(rec & 0xFFFFu); row = (int)(rec >> 16);     // (the word after the last row: the number of entries)
+            }
         } else {
             if (lane <= nrows) o = a.offsets[v0 + lane];
         }
@@ -556,7 +571,7 @@ struct WarpPipe {
             UnitBlock b{nullptr, 0u, 0, vi};
             if (q < total) {
                 if (e < ci) {
-                    const unsigned p = a.perm[oi + e];
+                    const unsigned p = a.compact ? reinterpret_cast<const unsigned short*>(a.perm)[oi + e] : a.perm[oi + e];
                     if (p < (unsigned)a.n_total) {
                         b.src = row_address(p) + cb;
                         b.bytes = (unsigned)(wcols * (long long)sizeof(VT));
@@ -592,7 +607,10 @@ struct WarpPipe {
         const unsigned span = n_valid >= 32 ? 0xFFFFFFFFu : ((1u << n_valid) - 1u);
         const unsigned want = ~(tabs.named[r0 >> 5] >> (r0 & 31)) & span;
         const int n = __popc(want);
-        if (n == 0) return true;
+        if (n == 0) {                                     // every row of the item is named: nothing to copy
+            if (lane == 0) polled = *reinterpret_cast<volatile int*>(&a.hdr->tables_ready);
+            return true;
+        }
         const long long cb = (long long)cblk * a.W;
         const long long wcols = min((long long)a.W, a.d - cb);
         const unsigned bytes = (unsigned)(wcols * (long long)sizeof(OT));
@@ -616,6 +634,8 @@ struct WarpPipe {
                     if (a.dense_in) { b.src = static_cast<const OT*>(a.dense_in) + at; b.bytes = bytes; }
                 }
             }
+            // the unit during which the last copies of the item are issued asks for the flag
+            if (base + 32 >= total && q == max(base, total - 1 - ns)) b.kind |= kUnitPoll;
             if (!run_block(acc, b, min(32, total - base), cblk)) return false;
         }
         return true;
@@ -696,23 +716,26 @@ struct WarpPipe {
         unsigned n_copy = 0;
         if constexpr (OVERLAP) {
             // Until the index cluster says its tables are complete: copy items.  The flag is asked for
-            // before an item and looked at after it, so the trip to memory costs nothing.
+            // while the last copies of an item are under way and looked at after the item, so the trip
+            // to memory costs nothing.
             n_copy = (unsigned)((a.vocab + a.copy_rows - 1) / a.copy_rows) * (unsigned)a.ncb;
+            ns = a.copy_slots;
             claim_begin(copies, &a.hdr->copy_counter, n_copy, true);
             volatile int* ready_flag = &a.hdr->tables_ready;
             bool ready = false;
             while (ok && !ready) {
                 int f = 0;
                 bool waited = false;
-                if (lane == 0) f = *ready_flag;
                 if (copies.item < n_copy) {
                     ok = do_copy(copies.item);
+                    f = polled;
                     claim_next(copies);
                 } else {
                     // nothing left to copy: wait for the tables, within the limit
                     waited = true;
                     if (lane == 0) {
                         const long long start = clock64();
+                        f = *ready_flag;
                         while (!f) {
                             if (*abort_flag || clock64() - start > kWaitCycles) break;
                             __nanosleep(200);
@@ -728,6 +751,7 @@ struct WarpPipe {
                 ok = load_tables_once();
             }
         }
+        if constexpr (OVERLAP) { ns = a.n_slots; islot = cslot = 0; }      // the ring is empty between items
         if (ok) {
             const unsigned n_chunks = (unsigned)a.hdr->n_chunks;
             const unsigned n_base = n_chunks + (unsigned)a.hdr->n_batches;
@@ -742,6 +766,7 @@ struct WarpPipe {
             }
         }
         if constexpr (OVERLAP) {
+            ns = a.copy_slots; islot = cslot = 0;
             while (ok && copies.item < n_copy) {      // the copy items that are left
                 ok = do_copy(copies.item);
                 claim_next(copies);
@@ -884,6 +909,12 @@ static cudaError_t launch_pipe_as(MainArgs a, int sm_count, cudaStream_t stream)
     const long long per_slot = (long long)grid * kPipeWarps * a.slot_bytes;
     long long slots = kInFlightBytes / per_slot;
     a.n_slots = (int)(slots < 2 ? 2 : (slots > kPipeSlots ? kPipeSlots : slots));
+    if (OVERLAP) {
+        // the same ring depth for copy items and for the items that follow (six slots for the latter measured
+        // no better: those run in waves that are bound by bandwidth and by their dependent look-ups, not by
+        // the depth of one warp's ring)
+        a.copy_slots = a.n_slots;
+    }
     return launch_pdl(k_reduce_rows<VT, OT, K, APPLY, OVERLAP>, dim3(grid), dim3(kPipeThreads), smem_for(a.n_slots), stream, a);
 }
 
