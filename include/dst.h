@@ -288,6 +288,21 @@ int dst_bytes_report(const int64_t* n_rows_per_slice, int32_t R, int64_t d, int6
 void dst_profile_events(void* before, void* after);
 int64_t dst_kernel_launches(void);
 
+/*
+ * Diagnostic of the library's bounded device-side waits (the paper has no counterpart: its
+ * failure mode is a host that runs out of memory, Section 3).  Every wait a kernel of this
+ * library makes -- on a copy's completion barrier, on a flag another CTA sets -- gives up after
+ * a limit, raises DST_ERR_TIMEOUT in the workspace header, and the kernel returns; nothing
+ * hangs and nothing traps.  This call runs that give-up path by itself: one CTA waits, with the
+ * routine the row-reduction kernel uses, on a barrier that nobody ever arrives on, for at most
+ * limit_cycles SM clock cycles (0 < limit_cycles <= 2^31).  When the stream has run,
+ * result->status (device or pinned memory, optional) holds DST_ERR_TIMEOUT, and so does the
+ * first word of `workspace` (>= 256 bytes, 256-byte aligned, cleared by the call).  The context
+ * stays usable; a densify call that follows behaves as usual.
+ */
+int dst_selftest_wait_limit(int64_t limit_cycles, void* workspace, size_t workspace_bytes, dst_stream_t stream,
+                            dst_result_t* result);
+
 #ifdef __cplusplus
 }
 #endif

@@ -80,6 +80,7 @@ SYMBOLS = {
     "dst_host_staging_bytes": (_sz, [_i64, _i64, _i64, ctypes.POINTER(_Opts)]),
     "dst_densify_concat_host": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, _vp,
                                                ctypes.POINTER(_Opts), _vp, _sz, _vp, _sz, _vp]),
+    "dst_selftest_wait_limit": (ctypes.c_int, [_i64, _vp, _sz, _vp, _vp]),
     "dst_profile_events": (None, [_vp, _vp]),
     "dst_kernel_launches": (ctypes.c_int64, []),
     "dst_bytes_report": (ctypes.c_int, [ctypes.POINTER(_i64), _i32, _i64, _i64, ctypes.POINTER(_Opts),
@@ -160,6 +161,15 @@ def dst_profile_events(before=None, after=None) -> None:
 
 def dst_kernel_launches() -> int:
     return int(load_library().dst_kernel_launches())
+
+
+def dst_selftest_wait_limit(limit_cycles: int, workspace: torch.Tensor, result: Optional[torch.Tensor] = None,
+                            stream=None) -> None:
+    """Run the give-up path of the library's bounded device-side waits on its own (see ``include/dst.h``)."""
+    rc = load_library().dst_selftest_wait_limit(int(limit_cycles), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                _stream_handle(stream), _ptr(result))
+    if rc != 0:
+        raise DstError(rc, "dst_selftest_wait_limit")
 
 
 def dst_workspace_bytes(n_rows_total: int, R: int, d: int, vocab: int, index_dtype=torch.int64,

@@ -490,6 +490,17 @@ int dst_accumulate(const dst_grad_t* grads, int32_t n, int64_t d, int64_t vocab,
                         nullptr, nullptr, result);
 }
 
+int dst_selftest_wait_limit(int64_t limit_cycles, void* workspace, size_t workspace_bytes, dst_stream_t stream,
+                            dst_result_t* result) {
+    if (limit_cycles <= 0 || limit_cycles > kWaitCycles || !workspace || workspace_bytes < 256) return DST_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return DST_ERR_INVALID_ARG;
+    if (cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess) return DST_ERR_CUDA;
+    if (launch_selftest_wait(static_cast<WsHeader*>(workspace), result, (long long)limit_cycles, stream) != cudaSuccess)
+        return DST_ERR_CUDA;
+    ++g_launches;
+    return DST_OK;
+}
+
 int dst_bytes_report(const int64_t* n_rows_per_slice, int32_t R, int64_t d, int64_t vocab, const dst_opts_t* opts,
                      dst_bytes_report_t* report) {
     if (!opts_ok(opts)) return opts ? DST_ERR_UNSUPPORTED : DST_ERR_INVALID_ARG;

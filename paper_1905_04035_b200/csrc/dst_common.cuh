@@ -275,6 +275,7 @@ cudaError_t launch_sum_dense(const SumParams& p, int out_type, int sm_count, cud
 cudaError_t launch_iota(void* indices, long long n, int index_type, int sm_count, cudaStream_t stream);
 cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,
                                cudaStream_t stream);
+cudaError_t launch_selftest_wait(WsHeader* hdr, dst_result_t* result, long long limit, cudaStream_t stream);
 
 // Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor
 // in the stream is still running (once all of the predecessor's CTAs have called pdl_trigger), so the

@@ -143,12 +143,13 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
     return ok != 0;
 }
 // Bounded wait: gives up when the limit is reached or another thread has given up.
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag,
+                                          long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag || clock64() - start > kWaitCycles) return false;
+        if (*abort_flag || clock64() - start > limit) return false;
     }
 }
 // global -> this CTA's shared memory, 16-byte aligned on both sides, bytes % 16 == 0
@@ -946,6 +947,33 @@ static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaSt
     if (ps.K == 2) return launch_pipe<VT, OT, 2, APPLY>(a, sm_count, stream);
     if (ps.K == 4 || kMaxK == 4) return launch_pipe<VT, OT, 4, APPLY>(a, sm_count, stream);
     return launch_pipe<VT, OT, kMaxK, APPLY>(a, sm_count, stream);
+}
+
+// The give-up path of the bounded waits, on its own: one CTA waits on a barrier nobody arrives on, with
+// the limit the caller gives, and must come back with DST_ERR_TIMEOUT in the header and in `result`.
+__global__ void __launch_bounds__(kPipeThreads) k_selftest_wait(WsHeader* hdr, dst_result_t* result, long long limit) {
+    __shared__ unsigned long long bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_addr(&bar), 1u);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (!mbar_wait(smem_addr(&bar), 0u, &s_abort, limit)) {      // what WarpPipe::give_up does
+        raise_status(hdr, DST_ERR_TIMEOUT);
+        s_abort = 1;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && result) {
+        __threadfence();
+        result->status = *reinterpret_cast<volatile int*>(&hdr->status);
+    }
+}
+
+cudaError_t launch_selftest_wait(WsHeader* hdr, dst_result_t* result, long long limit, cudaStream_t stream) {
+    k_selftest_wait<<<1, kPipeThreads, 0, stream>>>(hdr, result, limit);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,

@@ -185,7 +185,7 @@ def test_dtype_pairs(vt, ot):
 
 
 # ---------------------------------------------------------------------------
-# the two index paths and the pre-filled output of the small-input path
+# the two index paths; small inputs, where the row kernel copies the unnamed rows beside the index cluster
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("n,vocab,R", [
     (65535, 65536, 1),      # largest input of the one-kernel index path
@@ -193,7 +193,7 @@ def test_dtype_pairs(vt, ot):
     (3000, 65537, 1),       # one more vocabulary row: general path
     (3000, 65536, 64),      # most slices the one-kernel path takes
     (3000, 65536, 65),      # one more slice: general path
-    (3000, 1000, 3),        # small path, more rows than vocabulary: nothing is pre-filled
+    (3000, 1000, 3),        # small, but more rows than vocabulary: general path
 ])
 def test_index_path_boundaries(n, vocab, R):
     ns = [n // R + (1 if r < n % R else 0) for r in range(R)]
@@ -206,8 +206,8 @@ def test_index_path_boundaries(n, vocab, R):
 
 @pytest.mark.parametrize("d,with_dense,in_place", [(64, True, False), (2056, True, False), (512, False, False),
                                                    (512, True, True), (4096, True, True)])
-def test_prefilled_output_small_inputs(d, with_dense, in_place):
-    # few rows against the vocabulary: most of out is written by the index kernel's extra clusters
+def test_small_inputs_unnamed_rows_are_copied(d, with_dense, in_place):
+    # few rows against the vocabulary: most rows of out are plain copies of dense_in (or zeros)
     vocab = 40000 if d <= 512 else 6000
     hot = lambda rng, k: np.where(rng.random(k) < 0.4, 7, rng.integers(0, vocab, size=k))
     w = _custom(vocab, d, [1500, 0, 700], idx_fn=hot, with_dense=with_dense, std=0.5)
@@ -220,7 +220,7 @@ def test_prefilled_output_small_inputs(d, with_dense, in_place):
         assert_parity(w, run)
 
 
-def test_prefilled_output_bf16_and_out_of_range():
+def test_small_inputs_bf16_and_out_of_range():
     vocab = 50000
     def idx(rng, k):
         ix = rng.integers(0, vocab, size=k)
@@ -300,3 +300,95 @@ def test_bytes_report_matches_oracle():
         want = oracle.bytes_report(ns, d, vocab, index_dtype=it, value_dtype=vt, out_dtype=ot)
         for k, v in want.items():
             assert got[k] == v or abs(got[k] - v) <= 1e-12 * abs(v), k
+
+
+# ---------------------------------------------------------------------------
+# branches and guarantees that the named workloads do not reach
+# ---------------------------------------------------------------------------
+def test_more_heavy_rows_than_the_shared_memory_table_holds():
+    # every one of 3000 rows is heavy (about 67 entries each against chunks of 32): the row-reduction kernel
+    # keeps the first chunk ids of at most 1024 heavy rows in shared memory and searches the global table beyond
+    vocab, d, n = 3000, 64, 200_000
+    w = _custom(vocab, d, [n], std=0.05)
+    run = run_library(w)
+    orc = assert_parity(w, run)
+    assert orc.n_unique == vocab and int(orc.counts.min()) > 32
+
+
+def test_nan_inf_and_negative_zero_propagate():
+    # IEEE propagation: a NaN or an infinity in a value row or in dense_in reaches exactly the output elements it
+    # belongs to; -0 + -0 stays -0 and an unnamed row keeps its dense_in bits
+    vocab, d = 500, 64
+    w = _custom(vocab, d, [3000], idx_fn=lambda rng, n: rng.integers(0, 300, size=n))     # rows 300.. are unnamed
+    v, dn, ix = w.values[0], w.dense_in, w.indices[0]
+    v[10, 3] = np.nan; v[11, 4] = np.inf; v[12, 5] = -np.inf
+    ix[20] = ix[11]; v[20, 4] = -np.inf                              # +inf and -inf meet in one output element: NaN
+    dn[7, 9] = np.nan; dn[450, 1] = np.inf; dn[451, 2] = -0.0        # rows 450, 451 are unnamed
+    rows0 = np.flatnonzero(ix == 42)
+    v[rows0, 17] = -0.0; dn[42, 17] = -0.0                           # only negative zeros meet: -0
+    run = run_library(w)
+    orc = oracle_of(w)
+    got = to_numpy_f64(run.out)
+    want = orc.acc
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    assert np.array_equal(np.isposinf(got), np.isposinf(want)) and np.array_equal(np.isneginf(got), np.isneginf(want))
+    fin = np.isfinite(want)
+    assert np.all(np.abs(got[fin] - want[fin]) <= 1e-5 * orc.mag[fin] + 1e-7)
+    assert np.isnan(got[ix[10], 3]) and np.isnan(got[ix[11], 4]) and np.isneginf(got[ix[12], 5]) and np.isnan(got[7, 9])
+    assert np.isposinf(got[450, 1])
+    bits = raw_bits(run.out)
+    assert bits[451, 2] == 0x80000000 and bits[42, 17] == 0x80000000
+    assert run.result["status"] == 0
+
+
+@pytest.mark.parametrize("name", ["tiny", "custom_general", "custom_bf16"])
+def test_nothing_is_written_beyond_the_buffers(name):
+    # guard words behind every buffer the library writes: out, unique_rows, counts, the result block and the workspace
+    if name == "tiny":
+        w = make_workload("tiny")
+    elif name == "custom_general":
+        hot = lambda rng, n: np.where(rng.random(n) < 0.5, 3, rng.integers(0, 2000, size=n))
+        w = _custom(2000, 136, [70000, 0, 9000], idx_fn=hot)          # general index path, heavy rows
+    else:
+        w = _custom(70000, 64, [5000], value_dtype="bf16", out_dtype="bf16", index_dtype="i32")   # three radix passes
+    from gpu_helpers import TORCH_DT
+    idt, vdt, odt = TORCH_DT[w.index_dtype], TORCH_DT[w.value_dtype], TORCH_DT[w.out_dtype]
+    guard = 64                                                       # guard elements of each buffer's own type
+    def guarded(n, dtype, fill):
+        t = torch.full((n + guard,), fill, dtype=dtype, device="cuda")
+        return t, t[:n]
+    cap = max(1, min(w.n_rows_total, w.vocab))
+    out_all, out = guarded(w.vocab * w.d, odt, 7.0)
+    uniq_all, uniq = guarded(cap, idt, -3)
+    cnt_all, cnt = guarded(cap, torch.int32, -3)
+    res_all, res = guarded(6, torch.int32, -3)
+    ws_bytes = dst.dst_workspace_bytes(w.n_rows_total, len(w.indices), w.d, w.vocab, idt, vdt, odt)
+    ws_all = torch.full((ws_bytes + 4096,), 0xA5, dtype=torch.uint8, device="cuda")
+    slices = [(to_device(i, w.index_dtype), to_device(v, w.value_dtype)) for i, v in zip(w.indices, w.values)]
+    dense = to_device(w.dense_in, w.out_dtype) if w.dense_in is not None else None
+    dst.dst_densify_concat(slices, w.d, w.vocab, dense, out.view(w.vocab, w.d), ws_all[:ws_bytes], uniq, cnt, res)
+    torch.cuda.synchronize()
+    assert bool((out_all[w.vocab * w.d:] == 7.0).all())
+    assert bool((uniq_all[cap:] == -3).all()) and bool((cnt_all[cap:] == -3).all()) and bool((res_all[6:] == -3).all())
+    assert bool((ws_all[ws_bytes:] == 0xA5).all())
+    orc = oracle_of(w)
+    nu = int(res[1])
+    assert nu == orc.n_unique and np.array_equal(uniq[:nu].cpu().numpy(), orc.unique_rows)
+    assert bool((uniq[nu:] == -3).all()) and bool((cnt[nu:] == -3).all())      # nor beyond the entries that exist
+    got = to_numpy_f64(out.view(w.vocab, w.d))
+    from gpu_helpers import tolerance
+    assert np.all(np.abs(got - orc.acc) <= tolerance(w, orc))
+
+
+def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    # the give-up path of the bounded device-side waits: nothing arrives on the barrier, the limit is 100,000 cycles
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    res = torch.zeros(6, dtype=torch.int32, device="cuda")
+    dst.dst_selftest_wait_limit(100_000, ws, res)
+    torch.cuda.synchronize()                                          # returns: the wait ended by itself
+    assert int(res[0]) == 5 and dst.dst_status_string(5).startswith("a bounded device-side wait gave up")
+    assert int(ws[:4].view(torch.int32)[0]) == 5                      # the status word of the workspace header
+    with pytest.raises(dst.DstError):
+        dst.dst_selftest_wait_limit(0, ws, res)
+    w = make_workload("tiny")                                         # and the next call is an ordinary one
+    assert_parity(w, run_library(w))

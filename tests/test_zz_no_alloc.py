@@ -71,3 +71,36 @@ def test_static_workspace_entry_point_refuses_shapes_beyond_its_array():
     assert e.value.status == 3
     torch.cuda.synchronize()
     assert not out.any()        # nothing was enqueued
+
+
+def test_static_workspace_entry_point_against_the_oracle_on_both_index_paths_without_allocating():
+    """Directly against the CPU oracle, on a shape that takes the one-cluster index path and on one that takes the
+    general path (vocabulary above 65536: memset of the library's array, three radix passes, look-back
+    descriptors), interleaved so each finds the other's leftovers -- and the device's free memory is the same
+    before and after every call: the caller was promised that nothing is allocated."""
+    import oracle
+    small = make_workload("tiny", seed=3)
+    rng = np.random.default_rng(5)
+    vocab, d, n = 70000, 64, 2000
+    idx = np.where(rng.random(n) < 0.3, 69999, rng.integers(0, vocab, size=n)).astype(np.int64)
+    val = rng.standard_normal((n, d)).astype(np.float32)
+    dense = rng.standard_normal((vocab, d)).astype(np.float32)
+    assert dst.dst_workspace_bytes(n, 1, d, vocab) <= binding.STATIC_WORKSPACE_BYTES
+    cases = [(small.indices[0], small.values[0], small.dense_in, small.vocab, small.d), (idx, val, dense, vocab, d)]
+    dev = [tuple(torch.from_numpy(a).cuda() for a in c[:3]) for c in cases]
+    outs = [torch.full((c[3], c[4]), float("nan"), device="cuda") for c in cases]
+    res = torch.zeros(6, dtype=torch.int32, device="cuda")
+    dst.dst_densify_static(*dev[0][:2], cases[0][4], cases[0][3], dev[0][2], outs[0], None, None, res)   # first call on the device
+    torch.cuda.synchronize()
+    for k in (1, 0, 1, 0):
+        c = cases[k]
+        outs[k].fill_(float("nan"))
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        dst.dst_densify_static(dev[k][0], dev[k][1], c[4], c[3], dev[k][2], outs[k], None, None, res)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+        orc = oracle.densify([c[0]], [c[1]], c[4], c[3], c[2])
+        got = outs[k].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - orc.acc) <= 1e-5 * orc.mag + 1e-7)
+        assert int(res[0]) == 0 and int(res[1]) == orc.n_unique
