@@ -149,6 +149,47 @@ int dst_densify_apply_sgd(const dst_slice_t* slices, int32_t R, int64_t d, int64
                           void* unique_rows, int32_t* counts, dst_result_t* result);
 
 /*
+ * The same fusion for the optimizers that keep state (Section 4: whatever optimizer the distributed
+ * wrapper is handed; Section 1 for training in reduced precision).  With g the dense gradient
+ *
+ *     g[v, c] = grad_scale * (dense_in[v, c] + sum of the value rows that name v)
+ *
+ *   DST_OPT_SGD       weight <- weight - lr * g
+ *   DST_OPT_MOMENTUM  state1 <- momentum * state1 + g;   weight <- weight - lr * state1
+ *   DST_OPT_ADAM      state1 <- beta1 * state1 + (1 - beta1) * g;   state2 <- beta2 * state2 + (1 - beta2) * g * g
+ *                     weight <- weight - lr * (state1 / (1 - beta1^step)) / (sqrt(state2 / (1 - beta2^step)) + eps)
+ *
+ * g is never written.  weight, state1 and state2 are [vocab, d] fp32 device tensors, updated in
+ * place; every row takes the step, named or not (with momentum or Adam a zero gradient still
+ * moves the state), and every row of each tensor is read once and written once.  value rows and
+ * dense_in have one type, fp32 or bf16 (opts->value_type == opts->out_type, otherwise
+ * DST_ERR_UNSUPPORTED): bf16 is the reduced-precision gradient, grad_scale the reciprocal of its
+ * loss scale (1 for unscaled gradients), applied to the fp32 sum.  All arithmetic is fp32; the
+ * gradient of a row is summed in the order dst_densify_concat uses, dense_in last.  weight must
+ * not be dense_in or a state tensor; state tensors a kind does not use may be NULL.  `optimizer`
+ * is a HOST struct read during the call.  All other arguments, the optional outputs and the
+ * error behaviour are those of dst_densify_concat.
+ */
+typedef enum { DST_OPT_SGD = 0, DST_OPT_MOMENTUM = 1, DST_OPT_ADAM = 2 } dst_optimizer_kind_t;
+typedef struct {
+    int32_t kind;     /* dst_optimizer_kind_t */
+    int32_t step;     /* DST_OPT_ADAM: the number t of this step, starting at 1 */
+    float lr;
+    float momentum;   /* DST_OPT_MOMENTUM */
+    float beta1;      /* DST_OPT_ADAM */
+    float beta2;
+    float eps;
+    float grad_scale; /* multiplies the summed gradient */
+    void* state1;     /* DST_OPT_MOMENTUM: the momentum buffer; DST_OPT_ADAM: the first moment */
+    void* state2;     /* DST_OPT_ADAM: the second moment */
+} dst_optimizer_t;
+
+int dst_densify_apply(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab,
+                      const void* dense_in, void* weight, const dst_optimizer_t* optimizer, dst_stream_t stream,
+                      const dst_opts_t* opts, void* workspace, size_t workspace_bytes,
+                      void* unique_rows, int32_t* counts, dst_result_t* result);
+
+/*
  * dst_densify without a caller-supplied workspace.  (The paper has no counterpart:
  * this entry point exists for the sake of callers, not of the method.)
  *

@@ -10,6 +10,9 @@ from .binding import (  # noqa: F401
     DST_ACC_PROPOSED,
     DST_ACC_SPARSE_AS_DENSE,
     DST_ACC_STOCK,
+    DST_OPT_ADAM,
+    DST_OPT_MOMENTUM,
+    DST_OPT_SGD,
     DST_STATUS,
     Densifier,
     DstError,
@@ -17,6 +20,7 @@ from .binding import (  # noqa: F401
     dst_accumulate_plan,
     dst_bytes_report,
     dst_densify,
+    dst_densify_apply,
     dst_densify_apply_sgd,
     dst_densify_concat,
     dst_densify_concat_host,

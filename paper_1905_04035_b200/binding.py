@@ -47,6 +47,12 @@ class _BytesReport(ctypes.Structure):
                 ("sparse_over_dense", ctypes.c_double), ("gather_all_over_dense", ctypes.c_double)]
 
 
+class _Optimizer(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("step", ctypes.c_int32), ("lr", ctypes.c_float), ("momentum", ctypes.c_float),
+                ("beta1", ctypes.c_float), ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
+                ("grad_scale", ctypes.c_float), ("state1", ctypes.c_void_p), ("state2", ctypes.c_void_p)]
+
+
 class _Grad(ctypes.Structure):
     _fields_ = [("kind", ctypes.c_int32), ("reserved", ctypes.c_int32), ("indices", ctypes.c_void_p),
                 ("values", ctypes.c_void_p), ("n_rows", ctypes.c_int64)]
@@ -61,6 +67,7 @@ class _AccumPlan(ctypes.Structure):
 RESULT_BYTES = ctypes.sizeof(_Result)
 DST_GRAD_DENSE, DST_GRAD_SLICES = 0, 1
 DST_ACC_STOCK, DST_ACC_PROPOSED, DST_ACC_SPARSE_AS_DENSE = 0, 1, 2
+DST_OPT_SGD, DST_OPT_MOMENTUM, DST_OPT_ADAM = 0, 1, 2
 DST_BRANCH = {0: "empty", 1: "pass-through", 2: "reduce", 3: "convert+reduce", 4: "gather"}
 
 # name -> (restype, argtypes); also the list of symbols the header declares
@@ -75,6 +82,8 @@ SYMBOLS = {
                                           ctypes.POINTER(_Opts), _vp, _sz, _vp, _vp, _vp]),
     "dst_densify_apply_sgd": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, ctypes.c_float, _vp,
                                              ctypes.POINTER(_Opts), _vp, _sz, _vp, _vp, _vp]),
+    "dst_densify_apply": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, ctypes.POINTER(_Optimizer), _vp,
+                                         ctypes.POINTER(_Opts), _vp, _sz, _vp, _vp, _vp]),
     "dst_densify_static": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i64, _vp, _vp, _vp, ctypes.POINTER(_Opts),
                                           _vp, _vp, _vp]),
     "dst_host_staging_bytes": (_sz, [_i64, _i64, _i64, ctypes.POINTER(_Opts)]),
@@ -269,6 +278,44 @@ def dst_densify_apply_sgd(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]], d
                                        _ptr(unique_rows), _ptr(counts), _ptr(result))
     if rc != 0:
         raise DstError(rc, "dst_densify_apply_sgd")
+
+
+def dst_densify_apply(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]], d: int, vocab: int,
+                      dense_in: Optional[torch.Tensor], weight: torch.Tensor, workspace: torch.Tensor, *,
+                      kind: int = DST_OPT_SGD, lr: float, momentum: float = 0.0, beta1: float = 0.9,
+                      beta2: float = 0.999, eps: float = 1e-8, step: int = 1, grad_scale: float = 1.0,
+                      state1: Optional[torch.Tensor] = None, state2: Optional[torch.Tensor] = None,
+                      unique_rows: Optional[torch.Tensor] = None, counts: Optional[torch.Tensor] = None,
+                      result: Optional[torch.Tensor] = None, stream=None,
+                      index_dtype: Optional[torch.dtype] = None, grad_dtype: Optional[torch.dtype] = None) -> None:
+    """Enqueue ``dst_densify_apply`` (include/dst.h): the optimizer step (SGD, momentum, Adam) on the fp32
+    ``weight`` with the gradient grad_scale * (dense_in + densified slices), fp32 or bf16 gradients."""
+    lib = load_library()
+    R = len(slices)
+    index_dtype = slices[0][0].dtype if R else (index_dtype or torch.int64)
+    grad_dtype = slices[0][1].dtype if R else (grad_dtype or (dense_in.dtype if dense_in is not None else torch.float32))
+    arr = (_Slice * max(R, 1))()
+    for r, (idx, val) in enumerate(slices):
+        if idx.dtype != index_dtype or val.dtype != grad_dtype:
+            raise TypeError("all slices must share the index dtype and the gradient dtype")
+        _check_slice(idx, val, d, weight.device)
+        arr[r].indices, arr[r].values, arr[r].n_rows = idx.data_ptr(), val.data_ptr(), idx.shape[0]
+    for name, t in (("weight", weight), ("state1", state1), ("state2", state2)):
+        if t is not None and (t.dtype != torch.float32 or t.numel() != vocab * d or not t.is_contiguous()):
+            raise ValueError("%s must be contiguous float32 [vocab, d]" % name)
+    if dense_in is not None and (dense_in.dtype != grad_dtype or dense_in.numel() != vocab * d
+                                 or not dense_in.is_contiguous()):
+        raise ValueError("dense_in must be contiguous [vocab, d] in the gradient dtype")
+    o = _opts(index_dtype, grad_dtype, grad_dtype)
+    opt = _Optimizer(int(kind), int(step), float(lr), float(momentum), float(beta1), float(beta2), float(eps),
+                     float(grad_scale), state1.data_ptr() if state1 is not None else None,
+                     state2.data_ptr() if state2 is not None else None)
+    with torch.cuda.device(weight.device):
+        rc = lib.dst_densify_apply(arr, R, d, vocab, _ptr(dense_in), _ptr(weight), ctypes.byref(opt), _stream_handle(stream),
+                                   ctypes.byref(o), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                   _ptr(unique_rows), _ptr(counts), _ptr(result))
+    if rc != 0:
+        raise DstError(rc, "dst_densify_apply")
 
 
 def dst_densify(indices: torch.Tensor, values: torch.Tensor, d: int, vocab: int,

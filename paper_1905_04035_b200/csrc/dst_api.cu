@@ -1,4 +1,5 @@
 // C ABI of the densify library: argument checks, workspace carving, kernel sequencing.
+#include <math.h>
 #include <string.h>
 
 #include <atomic>
@@ -39,10 +40,23 @@ static int sm_count() {
 static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
                         void* out, cudaStream_t stream, const dst_opts_t* opts, void* workspace,
                         size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result,
-                        bool apply = false, float lr = 0.f) {
+                        const dst_optimizer_t* optimizer = nullptr) {
     if (!opts_ok(opts)) return opts ? DST_ERR_UNSUPPORTED : DST_ERR_INVALID_ARG;
-    if (apply && (opts->value_type != DST_F32 || opts->out_type != DST_F32)) return DST_ERR_UNSUPPORTED;
-    if (apply && out && out == dense_in) return DST_ERR_INVALID_ARG;   // the weight is not its own gradient
+    const bool apply = optimizer != nullptr;
+    // with an optimizer `out` is the fp32 weight; value rows and dense_in share one type
+    if (apply && opts->value_type != opts->out_type) return DST_ERR_UNSUPPORTED;
+    if (apply && out && (out == dense_in || out == optimizer->state1 || out == optimizer->state2))
+        return DST_ERR_INVALID_ARG;                                    // the weight is not its own gradient or state
+    if (apply) {
+        const int k = optimizer->kind;
+        if (k != DST_OPT_SGD && k != DST_OPT_MOMENTUM && k != DST_OPT_ADAM) return DST_ERR_INVALID_ARG;
+        if (k != DST_OPT_SGD && vocab > 0 && d > 0 && !optimizer->state1) return DST_ERR_INVALID_ARG;
+        if (k == DST_OPT_ADAM && vocab > 0 && d > 0 && (!optimizer->state2 || optimizer->state2 == optimizer->state1))
+            return DST_ERR_INVALID_ARG;
+        if (k == DST_OPT_ADAM && (optimizer->step < 1 || !(optimizer->beta1 >= 0.f && optimizer->beta1 < 1.f) ||
+                                  !(optimizer->beta2 >= 0.f && optimizer->beta2 < 1.f)))
+            return DST_ERR_INVALID_ARG;
+    }
     if (R < 0 || d < 0 || vocab < 0 || (R > 0 && !slices)) return DST_ERR_INVALID_ARG;
     if (vocab > kMaxVocab) return DST_ERR_UNSUPPORTED;
     int64_t n_total = 0;
@@ -76,6 +90,7 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     const size_t smallest = dtype_size(opts->value_type) < dtype_size(opts->out_type) ? dtype_size(opts->value_type)
                                                                                       : dtype_size(opts->out_type);
     bool vector_ok = d % int64_t(16 / smallest) == 0 && aligned16(out) && aligned16(dense_in);
+    if (apply) vector_ok = vector_ok && aligned16(optimizer->state1) && aligned16(optimizer->state2);
     for (int r = 0; r < R && vector_ok; ++r)
         if (slices[r].n_rows > 0 && !aligned16(slices[r].values)) vector_ok = false;
 
@@ -102,7 +117,8 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         fp.chunk = L.chunk; fp.batch_units = L.batch_units; fp.bfirst = reinterpret_cast<int*>(batches);
         fp.nodecnt_words = int((L.off_batches - L.off_nodecnt) / 4);
         compact = true;
-        overlap = apply ? dense_in != nullptr : out != dense_in;
+        // (plain SGD without a dense partner leaves the rows nobody names alone; momentum and Adam move every row)
+        overlap = apply ? (dense_in != nullptr || optimizer->kind != DST_OPT_SGD) : out != dense_in;
         fp.urec = reinterpret_cast<unsigned*>(ws + L.off_urow);
         fp.bitmap = reinterpret_cast<unsigned*>(ws + L.off_bitmap);
         fp.bitmap_words = L.bitmap_words;
@@ -163,7 +179,19 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     a.bitmap = reinterpret_cast<const unsigned*>(ws + L.off_bitmap);
     a.bitmap_words = L.bitmap_words;
     a.copy_rows = 8; a.copy_slots = 0;     // set by the launcher
-    a.apply = apply ? 1 : 0; a.lr = lr;
+    a.apply = 0; a.lr = 0.f; a.grad_scale = 1.f; a.opt_a = a.opt_b = a.opt_eps = 0.f; a.opt_bc1 = a.opt_bc2 = 1.f;
+    a.state1 = a.state2 = nullptr;
+    if (apply) {
+        a.apply = optimizer->kind + 1;               // the kernels' numbering: 1 SGD, 2 momentum, 3 Adam
+        a.lr = optimizer->lr; a.grad_scale = optimizer->grad_scale;
+        a.state1 = optimizer->state1; a.state2 = optimizer->state2;
+        if (optimizer->kind == DST_OPT_MOMENTUM) a.opt_a = optimizer->momentum;
+        if (optimizer->kind == DST_OPT_ADAM) {
+            a.opt_a = optimizer->beta1; a.opt_b = optimizer->beta2; a.opt_eps = optimizer->eps;
+            a.opt_bc1 = float(1.0 / (1.0 - pow(double(optimizer->beta1), double(optimizer->step))));
+            a.opt_bc2 = float(1.0 / (1.0 - pow(double(optimizer->beta2), double(optimizer->step))));
+        }
+    }
     a.urec = reinterpret_cast<const unsigned*>(ws + L.off_urow);
     if (t_ev_before && cudaEventRecord(t_ev_before, stream) != cudaSuccess) return DST_ERR_CUDA;
     if (launch_reduce_rows(a, opts->value_type, opts->out_type, vector_ok, sm_count(), stream) != cudaSuccess)
@@ -254,8 +282,19 @@ int dst_densify_concat(const dst_slice_t* slices, int32_t R, int64_t d, int64_t 
 int dst_densify_apply_sgd(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
                           void* weight, float lr, dst_stream_t stream, const dst_opts_t* opts, void* workspace,
                           size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
+    if (opts_ok(opts) && (opts->value_type != DST_F32 || opts->out_type != DST_F32)) return DST_ERR_UNSUPPORTED;
+    dst_optimizer_t sgd{};
+    sgd.kind = DST_OPT_SGD; sgd.lr = lr; sgd.grad_scale = 1.f;
     return densify_impl(slices, R, d, vocab, dense_in, weight, stream, opts, workspace, workspace_bytes, unique_rows,
-                        counts, result, true, lr);
+                        counts, result, &sgd);
+}
+
+int dst_densify_apply(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
+                      void* weight, const dst_optimizer_t* optimizer, dst_stream_t stream, const dst_opts_t* opts,
+                      void* workspace, size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
+    if (!optimizer) return DST_ERR_INVALID_ARG;
+    return densify_impl(slices, R, d, vocab, dense_in, weight, stream, opts, workspace, workspace_bytes, unique_rows,
+                        counts, result, optimizer);
 }
 
 int dst_densify_static(const void* indices, const void* values, int64_t n_rows, int64_t d, int64_t vocab,

@@ -136,8 +136,14 @@ struct MainArgs {
     int ncb;         // column blocks per row
     int slot_bytes;
     int n_slots;
-    int apply;       // 1: `out` holds a weight and gets the SGD step (fp32 only), see dst_densify_apply_sgd
+    int apply;       // 0: `out` receives the gradient; 1 SGD, 2 momentum, 3 Adam: `out` is an fp32 weight that takes the step
     float lr;        // learning rate of that step
+    float grad_scale;           // the summed gradient is multiplied by this (reciprocal of the loss scale)
+    float opt_a, opt_b;         // momentum: mu, -; Adam: beta1, beta2
+    float opt_eps;              // Adam
+    float opt_bc1, opt_bc2;     // Adam: 1 / (1 - beta1^t), 1 / (1 - beta2^t)
+    void* state1;               // [vocab, d] fp32: momentum buffer / Adam's first moment
+    void* state2;               // [vocab, d] fp32: Adam's second moment
     int compact;     // the row batches list only the named rows (urow / uoff); the others are not this item list's business
     // Overlapped small-input path: the kernel starts beside the index cluster.  Until tables_ready it gives the rows
     // nobody names their dense_in row (copy items of copy_rows consecutive rows, named ones skipped by the bitmap),

@@ -31,6 +31,8 @@
 // when the index cluster flags its tables complete the warps turn to the chunk items and row
 // batches (which then list named rows only), and finish whatever copy items are left.  The two
 // kinds of item write disjoint rows, so no order between them is needed.
+#include <type_traits>
+
 #include "dst_common.cuh"
 
 namespace dst {
@@ -164,7 +166,9 @@ enum : int {
     kUnitFinal = 2,      // finish output row y (slot holds its dense_in row unless there is no dense_in)
     kUnitCopy = 4,       // with kUnitFinal: nobody names the row, out = dense_in bit for bit
     kUnitChunkEnd = 8,   // last entry of chunk y: store the partial row, climb the tree
-    kUnitPoll = 16       // (copy items) ask now whether the index cluster has finished; the answer is looked at after the item
+    kUnitPoll = 16,      // (copy items) ask now whether the index cluster has finished; the answer is looked at after the item
+    kUnitState1 = 32,    // optimizer step: the slot holds the row of state1 (momentum buffer / Adam's m) of output row y
+    kUnitState2 = 64     // optimizer step: ... of state2 (Adam's v)
 };
 
 constexpr int kTabCache = 64;       // slices whose table is copied into shared memory
@@ -187,11 +191,22 @@ struct UnitBlock {
     int y;               // output row (kUnitFinal) or chunk id (kUnitChunkEnd)
 };
 
-// APPLY: instead of writing the accumulated gradient, take the SGD step on the weight that `out` holds
-// (fp32 rows only): out <- out - lr * (dense_in + sum of value rows).
+// OPT: 0 writes the accumulated gradient; otherwise `out` holds an fp32 weight that takes an optimizer step
+// with the gradient g = grad_scale * (dense_in + sum of value rows), which is never written:
+//   kOptSgd       out <- out - lr * g
+//   kOptMomentum  b <- mu * b + g;  out <- out - lr * b                                  (b: state1)
+//   kOptAdam      m <- beta1 * m + (1 - beta1) * g;  v <- beta2 * v + (1 - beta2) * g * g  (m: state1, v: state2)
+//                 out <- out - lr * (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps)
+// The rows of the state ride the ring as further closing units of an output row (v, then m, then the
+// weight), each read once and written once.  value rows and dense_in have one type (fp32 or bf16);
+// weight and state are fp32.
 // OVERLAP: the kernel runs beside the index cluster and starts with copy items (small inputs, see above).
-template <typename VT, typename OT, int K, bool APPLY = false, bool OVERLAP = false>
+enum : int { kOptNone = 0, kOptSgd = 1, kOptMomentum = 2, kOptAdam = 3 };
+
+template <typename VT, typename OT, int K, int OPT = kOptNone, bool OVERLAP = false>
 struct WarpPipe {
+    static constexpr bool APPLY = OPT != kOptNone;
+    using WT = std::conditional_t<APPLY, float, OT>;     // what `out` holds
     static constexpr int VC = 16 / sizeof(VT);     // columns per 16-byte group of a value row
     const MainArgs& a;
     const int lane;
@@ -207,6 +222,7 @@ struct WarpPipe {
     unsigned issued_mask;     // slots with a copy that may still be in flight
     int polled;               // lane 0: tables_ready as last asked for (kUnitPoll)
     int ns;                   // slots of the ring in use (<= a.n_slots, the slots there are); changed only when the ring is empty
+    Acc<VC> aux[K];           // kOptAdam: sqrt(vhat) + eps of the row being closed, between its v unit and its m unit
 
     __device__ WarpPipe(const MainArgs& args, unsigned ring_addr, unsigned bar_addr, char* ring_generic, volatile int* ab,
                         CtaTables& t)
@@ -214,6 +230,65 @@ struct WarpPipe {
           cslot(0), cphase(0u), issued_mask(0u), polled(0), ns(args.n_slots) {}
 
     __device__ __forceinline__ int col(int k) const { return (k * 32 + lane) * VC; }
+
+    // The optimizer's arithmetic on one column group.  `g` comes in as the raw sum (dense_in + value rows).
+    // state unit of kOptMomentum: s holds b; leaves the new b in s and in g (what the weight unit subtracts)
+    __device__ __forceinline__ void step_momentum(Acc<VC>& g, Acc<VC>& s) const {
+#pragma unroll
+        for (int i = 0; i < VC; ++i) { s.x[i] = fmaf(a.opt_a, s.x[i], a.grad_scale * g.x[i]); g.x[i] = s.x[i]; }
+    }
+    // first state unit of kOptAdam: s holds v; leaves the new v in s, the scaled gradient in g, the denominator in den
+    __device__ __forceinline__ void step_adam_v(Acc<VC>& g, Acc<VC>& s, Acc<VC>& den) const {
+#pragma unroll
+        for (int i = 0; i < VC; ++i) {
+            g.x[i] = a.grad_scale * g.x[i];
+            s.x[i] = fmaf(a.opt_b, s.x[i], (1.f - a.opt_b) * (g.x[i] * g.x[i]));
+            den.x[i] = sqrtf(s.x[i] * a.opt_bc2) + a.opt_eps;
+        }
+    }
+    // second state unit of kOptAdam: s holds m; leaves the new m in s and the bias-corrected step direction in g
+    __device__ __forceinline__ void step_adam_m(Acc<VC>& g, Acc<VC>& s, const Acc<VC>& den) const {
+#pragma unroll
+        for (int i = 0; i < VC; ++i) {
+            s.x[i] = fmaf(a.opt_a, s.x[i], (1.f - a.opt_a) * g.x[i]);
+            g.x[i] = (s.x[i] * a.opt_bc1) / den.x[i];
+        }
+    }
+    // the weight unit: w holds the weight row; g what the state units left (kOptSgd: the raw sum)
+    __device__ __forceinline__ void step_weight(const Acc<VC>& g, Acc<VC>& w) const {
+#pragma unroll
+        for (int i = 0; i < VC; ++i) w.x[i] = fmaf(-a.lr, OPT == kOptSgd ? a.grad_scale * g.x[i] : g.x[i], w.x[i]);
+    }
+    // The units that close an output row, in ring order: its dense_in row (OPT: one more row to add), then,
+    // with an optimizer, Adam's v row, the m / momentum row and last the weight row.
+    __device__ __forceinline__ int n_closing() const {
+        if constexpr (!APPLY) return 1;
+        return (a.dense_in ? 1 : 0) + (OPT == kOptAdam ? 2 : (OPT == kOptMomentum ? 1 : 0)) + 1;
+    }
+    __device__ __forceinline__ void closing_unit(UnitBlock& b, int c, long long at, long long wcols, bool named) const {
+        if constexpr (APPLY) {
+            const unsigned fbytes = (unsigned)(wcols * 4);
+            if (a.dense_in) {
+                if (c == 0) { b.src = static_cast<const OT*>(a.dense_in) + at; b.bytes = (unsigned)(wcols * (long long)sizeof(OT)); b.kind = kUnitAdd; return; }
+                --c;
+            }
+            if constexpr (OPT == kOptAdam) {
+                if (c == 0) { b.src = static_cast<const float*>(a.state2) + at; b.bytes = fbytes; b.kind = kUnitState2; return; }
+                --c;
+            }
+            if constexpr (OPT == kOptAdam || OPT == kOptMomentum) {
+                if (c == 0) { b.src = static_cast<const float*>(a.state1) + at; b.bytes = fbytes; b.kind = kUnitState1; return; }
+                --c;
+            }
+            b.src = static_cast<const float*>(a.out) + at; b.bytes = fbytes; b.kind = kUnitFinal;
+        } else {
+            b.kind = kUnitFinal | (named ? 0 : kUnitCopy);
+            if (a.dense_in) { b.src = static_cast<const OT*>(a.dense_in) + at; b.bytes = (unsigned)(wcols * (long long)sizeof(OT)); }
+        }
+    }
+    __device__ __forceinline__ float* state_row(int which, int y, long long cb) const {
+        return static_cast<float*>(which == 1 ? a.state1 : a.state2) + (long long)y * a.d + cb;
+    }
 
     // unit j of the block goes into the next slot
     __device__ __forceinline__ void issue(const UnitBlock& b, int j) {
@@ -379,7 +454,7 @@ struct WarpPipe {
             if (!last) return true;
             __threadfence();
             const bool root = n_parent == 1;
-            // fp32 rows in, fp32 rows out: the root's dense row rides the ring behind the children
+            // fp32 rows in, fp32 dense rows: the root's dense row rides the ring behind the children
             constexpr bool kDenseInRing = sizeof(VT) == 4 && sizeof(OT) == 4;
             const float* dense_row = nullptr;
             if constexpr (kDenseInRing)
@@ -390,8 +465,52 @@ struct WarpPipe {
                 // The output may be the dense input itself, so the compiler keeps loads and stores in
                 // program order: read the whole dense row first, then store, or every column group
                 // pays its own trip to memory.
-                const OT* din = APPLY ? static_cast<const OT*>(a.out)            // the weight row
-                                      : (kDenseInRing ? nullptr : static_cast<const OT*>(a.dense_in));
+                if constexpr (APPLY) {
+                    // weight and state rows straight from memory (heavy rows are few): all loads of a step first
+                    float* wrow = static_cast<float*>(a.out) + (long long)hi.row * a.d + cb;
+                    if constexpr (!kDenseInRing) {
+                        if (a.dense_in) {
+                            const OT* drow = static_cast<const OT*>(a.dense_in) + (long long)hi.row * a.d + cb;
+                            Acc<VC> dn[K];
+#pragma unroll
+                            for (int k = 0; k < K; ++k) { zero(dn[k]); if (col(k) < wcols) load_elems(drow + col(k), dn[k]); }
+#pragma unroll
+                            for (int k = 0; k < K; ++k) add(acc[k], dn[k]);
+                        }
+                    }
+                    if constexpr (OPT == kOptMomentum || OPT == kOptAdam) {
+                        float* srow = state_row(OPT == kOptAdam ? 2 : 1, hi.row, cb);
+                        Acc<VC> st[K];
+#pragma unroll
+                        for (int k = 0; k < K; ++k) { zero(st[k]); if (col(k) < wcols) load_elems(srow + col(k), st[k]); }
+#pragma unroll
+                        for (int k = 0; k < K; ++k) {
+                            if constexpr (OPT == kOptAdam) step_adam_v(acc[k], st[k], aux[k]); else step_momentum(acc[k], st[k]);
+                            if (col(k) < wcols) store_out(srow + col(k), st[k]);
+                        }
+                    }
+                    if constexpr (OPT == kOptAdam) {
+                        float* srow = state_row(1, hi.row, cb);
+                        Acc<VC> st[K];
+#pragma unroll
+                        for (int k = 0; k < K; ++k) { zero(st[k]); if (col(k) < wcols) load_elems(srow + col(k), st[k]); }
+#pragma unroll
+                        for (int k = 0; k < K; ++k) {
+                            step_adam_m(acc[k], st[k], aux[k]);
+                            if (col(k) < wcols) store_out(srow + col(k), st[k]);
+                        }
+                    }
+                    Acc<VC> wt[K];
+#pragma unroll
+                    for (int k = 0; k < K; ++k) { zero(wt[k]); if (col(k) < wcols) load_elems(wrow + col(k), wt[k]); }
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        step_weight(acc[k], wt[k]);
+                        if (col(k) < wcols) store_out(wrow + col(k), wt[k]);
+                    }
+                    return true;
+                }
+                const OT* din = kDenseInRing ? nullptr : static_cast<const OT*>(a.dense_in);
                 OT* out = static_cast<OT*>(a.out) + (long long)hi.row * a.d + cb;
                 constexpr int KH = (sizeof(VT) == 2 && K >= 4) ? K / 2 : K;
 #pragma unroll
@@ -406,12 +525,7 @@ struct WarpPipe {
 #pragma unroll
                     for (int k = 0; k < KH; ++k) {
                         const int c = col(h0 + k);
-                        if constexpr (APPLY) {
-#pragma unroll
-                            for (int i = 0; i < VC; ++i) acc[h0 + k].x[i] = fmaf(-a.lr, acc[h0 + k].x[i], dn[k].x[i]);
-                        } else {
-                            add(acc[h0 + k], dn[k]);
-                        }
+                        add(acc[h0 + k], dn[k]);
                         if (c < wcols) store_out(out + c, acc[h0 + k]);
                     }
                 }
@@ -440,7 +554,7 @@ struct WarpPipe {
     __device__ bool run_block(Acc<VC> (&acc)[K], const UnitBlock& b, int n, int cblk) {
         const long long cb = (long long)cblk * a.W;
         const int wcols = (int)min((long long)a.W, a.d - cb);
-        OT* const out = static_cast<OT*>(a.out);
+        WT* const out = static_cast<WT*>(a.out);
         const int ahead = min(n, ns);
         for (int j = 0; j < ahead; ++j) issue(b, j);
         for (int j = 0; j < n; ++j) {
@@ -463,22 +577,43 @@ struct WarpPipe {
 #pragma unroll
                 for (int k = 0; k < K; ++k) add(acc[k], v[k]);
             }
+            if constexpr (OPT == kOptMomentum || OPT == kOptAdam) {
+                if (kind & (kUnitState1 | kUnitState2)) {
+                    // the slot holds a row of optimizer state: update it, keep what the next closing unit needs
+                    float* srow = state_row((kind & kUnitState1) ? 1 : 2, y, cb);
+                    Acc<VC> st[K];
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        const int c = col(k);
+                        zero(st[k]);
+                        if (c < wcols) load_elems(reinterpret_cast<const float*>(sp) + c, st[k]);
+                    }
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        const int c = col(k);
+                        if constexpr (OPT == kOptMomentum) {
+                            step_momentum(acc[k], st[k]);
+                        } else {
+                            if (kind & kUnitState2) step_adam_v(acc[k], st[k], aux[k]); else step_adam_m(acc[k], st[k], aux[k]);
+                        }
+                        if (c < wcols) store_out(srow + c, st[k]);
+                    }
+                }
+            }
             if (kind & kUnitFinal) {
-                OT* orow = out + (long long)y * a.d + cb;
+                WT* orow = out + (long long)y * a.d + cb;
                 Acc<VC> dn[K];                            // the dense row first, all of it, then the stores
 #pragma unroll
                 for (int k = 0; k < K; ++k) {
                     const int c = col(k);
                     zero(dn[k]);
-                    if ((APPLY || a.dense_in) && c < wcols) load_elems(reinterpret_cast<const OT*>(sp) + c, dn[k]);
+                    if ((APPLY || a.dense_in) && c < wcols) load_elems(reinterpret_cast<const WT*>(sp) + c, dn[k]);
                 }
 #pragma unroll
                 for (int k = 0; k < K; ++k) {
                     const int c = col(k);
                     if constexpr (APPLY) {
-                        // the slot holds the weight row; acc holds the whole gradient of the row
-#pragma unroll
-                        for (int i = 0; i < VC; ++i) dn[k].x[i] = fmaf(-a.lr, acc[k].x[i], dn[k].x[i]);
+                        step_weight(acc[k], dn[k]);       // the slot holds the weight row
                     } else {
                         if (!(kind & kUnitCopy)) add(dn[k], acc[k]);
                     }
@@ -545,9 +680,7 @@ struct WarpPipe {
         }
         const int o_next = __shfl_down_sync(0xFFFFFFFFu, o, 1);
         const int cnt = lane < nrows ? o_next - o : 0;
-        // APPLY: the dense row is one more unit to add, before the weight row closes the row
-        const bool dense_unit = APPLY && a.dense_in;
-        const int nunits = (lane < nrows && cnt <= a.chunk) ? cnt + 1 + (dense_unit ? 1 : 0) : 0;   // heavy rows belong to the chunk items
+        const int nunits = (lane < nrows && cnt <= a.chunk) ? cnt + n_closing() : 0;   // heavy rows belong to the chunk items
         int incl = nunits;
 #pragma unroll
         for (int s = 1; s < 32; s <<= 1) {
@@ -578,19 +711,8 @@ struct WarpPipe {
                         b.bytes = (unsigned)(wcols * (long long)sizeof(VT));
                         b.kind = kUnitAdd;
                     }
-                } else if (dense_unit && e == ci) {
-                    b.src = static_cast<const OT*>(a.dense_in) + (long long)b.y * a.d + cb;
-                    b.bytes = (unsigned)(wcols * (long long)sizeof(OT));
-                    b.kind = kUnitAdd;
                 } else {
-                    b.kind = kUnitFinal | (ci == 0 ? kUnitCopy : 0);
-                    if constexpr (APPLY) {
-                        b.src = static_cast<const OT*>(a.out) + (long long)b.y * a.d + cb;
-                        b.bytes = (unsigned)(wcols * (long long)sizeof(OT));
-                    } else if (a.dense_in) {
-                        b.src = static_cast<const OT*>(a.dense_in) + (long long)b.y * a.d + cb;
-                        b.bytes = (unsigned)(wcols * (long long)sizeof(OT));
-                    }
+                    closing_unit(b, e - ci, (long long)b.y * a.d + cb, wcols, ci != 0);
                 }
             }
             if (!run_block(acc, b, min(32, total - base), cblk)) return false;
@@ -614,26 +736,17 @@ struct WarpPipe {
         }
         const long long cb = (long long)cblk * a.W;
         const long long wcols = min((long long)a.W, a.d - cb);
-        const unsigned bytes = (unsigned)(wcols * (long long)sizeof(OT));
         Acc<VC> acc[K];
 #pragma unroll
         for (int k = 0; k < K; ++k) zero(acc[k]);
-        const int per_row = APPLY ? 2 : 1;
+        const int per_row = n_closing();
         const int total = n * per_row;
         for (int base = 0; base < total; base += 32) {
             const int q = base + lane;
             UnitBlock b{nullptr, 0u, 0, 0};
             if (q < total) {
                 b.y = r0 + (int)__fns(want, 0u, q / per_row + 1);          // the (q / per_row + 1)-th row that is wanted
-                const long long at = (long long)b.y * a.d + cb;
-                if (APPLY && !(q & 1)) {
-                    b.src = static_cast<const OT*>(a.dense_in) + at; b.bytes = bytes; b.kind = kUnitAdd;
-                } else if (APPLY) {
-                    b.src = static_cast<const OT*>(a.out) + at; b.bytes = bytes; b.kind = kUnitFinal;
-                } else {
-                    b.kind = kUnitFinal | kUnitCopy;
-                    if (a.dense_in) { b.src = static_cast<const OT*>(a.dense_in) + at; b.bytes = bytes; }
-                }
+                closing_unit(b, q % per_row, (long long)b.y * a.d + cb, wcols, false);
             }
             // the unit during which the last copies of the item are issued asks for the flag
             if (base + 32 >= total && q == max(base, total - 1 - ns)) b.kind |= kUnitPoll;
@@ -785,8 +898,8 @@ struct WarpPipe {
     }
 };
 
-template <typename VT, typename OT, int K, bool APPLY = false, bool OVERLAP = false>
-__global__ void __launch_bounds__(kPipeThreads, sizeof(VT) == 2 ? 4 : 2)
+template <typename VT, typename OT, int K, int OPT = kOptNone, bool OVERLAP = false>
+__global__ void __launch_bounds__(kPipeThreads, (sizeof(VT) == 2 && OPT == kOptNone) ? 4 : 2)
 k_reduce_rows(const __grid_constant__ MainArgs a) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ int s_abort;
@@ -843,7 +956,7 @@ k_reduce_rows(const __grid_constant__ MainArgs a) {
     __syncthreads();
     {
         char* my_ring = slot_base + (size_t)warp * (size_t)a.n_slots * (size_t)a.slot_bytes;
-        WarpPipe<VT, OT, K, APPLY, OVERLAP> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort, tabs);
+        WarpPipe<VT, OT, K, OPT, OVERLAP> pipe(a, smem_addr(my_ring), smem_addr(&bar_base[warp * a.n_slots]), my_ring, &s_abort, tabs);
         // after a failed wait in an earlier kernel the tables are not to be trusted: touch nothing
         if (OVERLAP ? !s_abort : *reinterpret_cast<volatile int*>(&a.hdr->status) != DST_ERR_TIMEOUT) pipe.run();
     }
@@ -859,7 +972,8 @@ k_reduce_rows(const __grid_constant__ MainArgs a) {
     }
 }
 
-// Any d, any alignment: one thread per output element, segment summed in order.
+// Any d, any alignment: one thread per output element, segment summed in order.  With an optimizer
+// (a.apply != 0) `out` is the fp32 weight and the state tensors take their step too.
 template <typename VT, typename OT>
 __global__ void __launch_bounds__(256)
 k_reduce_rows_scalar(const MainArgs a) {
@@ -868,19 +982,33 @@ k_reduce_rows_scalar(const MainArgs a) {
     if (blockIdx.x == 0 && threadIdx.x == 0 && a.result) a.result->status = status;
     if (status == DST_ERR_TIMEOUT) return;     // a wait gave up in an earlier kernel: the tables are not to be trusted
     const OT* din = static_cast<const OT*>(a.dense_in);
-    OT* out = static_cast<OT*>(a.out);
     for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
         const int v = (int)(e / a.d);
         const long long c = e - (long long)v * a.d;
         const int beg = max(a.offsets[v], 0), end = min(a.offsets[v + 1], a.n_total);
-        if (beg >= end && !a.apply) { out[e] = din ? din[e] : OT(0.f); continue; }
+        if (beg >= end && !a.apply) { static_cast<OT*>(a.out)[e] = din ? din[e] : OT(0.f); continue; }
         float acc = 0.f;
         for (int j = beg; j < end; ++j) {
             unsigned p = a.perm[j];
             if (p < (unsigned)a.n_total) acc += (float)resolve_row<VT>(a, p)[c];
         }
         if (din) acc += (float)din[e];
-        out[e] = a.apply ? OT(fmaf(-a.lr, acc, (float)out[e])) : OT(acc);
+        if (!a.apply) { static_cast<OT*>(a.out)[e] = OT(acc); continue; }
+        float* w = static_cast<float*>(a.out) + e;
+        float g = a.grad_scale * acc;
+        if (a.apply == kOptMomentum) {
+            float* b = static_cast<float*>(a.state1) + e;
+            g = fmaf(a.opt_a, *b, g);
+            *b = g;
+        } else if (a.apply == kOptAdam) {
+            float* m = static_cast<float*>(a.state1) + e;
+            float* vv = static_cast<float*>(a.state2) + e;
+            const float v2 = fmaf(a.opt_b, *vv, (1.f - a.opt_b) * (g * g));
+            const float m2 = fmaf(a.opt_a, *m, (1.f - a.opt_a) * g);
+            *vv = v2; *m = m2;
+            g = (m2 * a.opt_bc1) / (sqrtf(v2 * a.opt_bc2) + a.opt_eps);
+        }
+        *w = fmaf(-a.lr, g, *w);
     }
 }
 
@@ -889,19 +1017,19 @@ k_reduce_rows_scalar(const MainArgs a) {
 // index lookup, a node of a combine tree), which is what a short call is made of.
 constexpr long long kInFlightBytes = 14ll << 20;
 
-template <typename VT, typename OT, int K, bool APPLY, bool OVERLAP>
+template <typename VT, typename OT, int K, int OPT, bool OVERLAP>
 static cudaError_t launch_pipe_as(MainArgs a, int sm_count, cudaStream_t stream) {
     auto smem_for = [&](int slots) { return size_t(kPipeHeaderReserve) + size_t(kPipeWarps) * size_t(slots) * size_t(a.slot_bytes); };
     // the shared-memory opt-in and the occupancy answer are asked of the runtime once per device and variant
     static SmemOptIn opt_in;
     static std::atomic<int> resident_on[64];
-    cudaError_t e = ensure_dynamic_smem(k_reduce_rows<VT, OT, K, APPLY, OVERLAP>, smem_for(kPipeSlots), opt_in);
+    cudaError_t e = ensure_dynamic_smem(k_reduce_rows<VT, OT, K, OPT, OVERLAP>, smem_for(kPipeSlots), opt_in);
     if (e != cudaSuccess) return e;
     int dev = -1, resident = 0;                          // CTAs of this variant an SM holds with full rings
     const bool cached = cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64;
     if (cached) resident = resident_on[dev].load();
     if (resident < 1) {
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, k_reduce_rows<VT, OT, K, APPLY, OVERLAP>, kPipeThreads, smem_for(kPipeSlots));
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, k_reduce_rows<VT, OT, K, OPT, OVERLAP>, kPipeThreads, smem_for(kPipeSlots));
         if (e != cudaSuccess) return e;
         if (resident < 1) return cudaErrorLaunchOutOfResources;
         if (cached) resident_on[dev].store(resident);
@@ -916,16 +1044,16 @@ static cudaError_t launch_pipe_as(MainArgs a, int sm_count, cudaStream_t stream)
         // the depth of one warp's ring)
         a.copy_slots = a.n_slots;
     }
-    return launch_pdl(k_reduce_rows<VT, OT, K, APPLY, OVERLAP>, dim3(grid), dim3(kPipeThreads), smem_for(a.n_slots), stream, a);
+    return launch_pdl(k_reduce_rows<VT, OT, K, OPT, OVERLAP>, dim3(grid), dim3(kPipeThreads), smem_for(a.n_slots), stream, a);
 }
 
-template <typename VT, typename OT, int K, bool APPLY>
+template <typename VT, typename OT, int K, int OPT>
 static cudaError_t launch_pipe(const MainArgs& a, int sm_count, cudaStream_t stream) {
-    return a.overlap ? launch_pipe_as<VT, OT, K, APPLY, true>(a, sm_count, stream)
-                     : launch_pipe_as<VT, OT, K, APPLY, false>(a, sm_count, stream);
+    return a.overlap ? launch_pipe_as<VT, OT, K, OPT, true>(a, sm_count, stream)
+                     : launch_pipe_as<VT, OT, K, OPT, false>(a, sm_count, stream);
 }
 
-template <typename VT, typename OT, bool APPLY = false>
+template <typename VT, typename OT, int OPT = kOptNone>
 static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaStream_t stream) {
     if (!vector_ok) {
         long long total = (long long)a.vocab * a.d;
@@ -935,18 +1063,19 @@ static cudaError_t launch_typed(MainArgs a, bool vector_ok, int sm_count, cudaSt
         k_reduce_rows_scalar<VT, OT><<<(int)blocks, 256, 0, stream>>>(a);
         return cudaGetLastError();
     }
-    const PipeShape ps = pipe_shape((int)sizeof(VT), (int)sizeof(OT), a.d);
+    // slots hold value rows, dense_in rows and, with an optimizer, fp32 weight and state rows
+    const PipeShape ps = pipe_shape((int)sizeof(VT), OPT != kOptNone ? 4 : (int)sizeof(OT), a.d);
     a.W = ps.W; a.ncb = ps.ncb; a.slot_bytes = ps.slot_bytes; a.n_slots = ps.n_slots;
     {
         // a copy item: about 32 KB worth of consecutive rows, 8 to 32 of them
-        const long long row_bytes = (long long)ps.W * (long long)sizeof(OT);
+        const long long row_bytes = (long long)ps.W * (OPT != kOptNone ? 4ll : (long long)sizeof(OT));
         a.copy_rows = row_bytes * 32 <= 32768 ? 32 : (row_bytes * 16 <= 32768 ? 16 : 8);
     }
     constexpr int kMaxK = sizeof(VT) == 4 ? 8 : 4;
-    if (ps.K == 1) return launch_pipe<VT, OT, 1, APPLY>(a, sm_count, stream);
-    if (ps.K == 2) return launch_pipe<VT, OT, 2, APPLY>(a, sm_count, stream);
-    if (ps.K == 4 || kMaxK == 4) return launch_pipe<VT, OT, 4, APPLY>(a, sm_count, stream);
-    return launch_pipe<VT, OT, kMaxK, APPLY>(a, sm_count, stream);
+    if (ps.K == 1) return launch_pipe<VT, OT, 1, OPT>(a, sm_count, stream);
+    if (ps.K == 2) return launch_pipe<VT, OT, 2, OPT>(a, sm_count, stream);
+    if (ps.K == 4 || kMaxK == 4) return launch_pipe<VT, OT, 4, OPT>(a, sm_count, stream);
+    return launch_pipe<VT, OT, kMaxK, OPT>(a, sm_count, stream);
 }
 
 // The give-up path of the bounded waits, on its own: one CTA waits on a barrier nobody arrives on, with
@@ -979,8 +1108,18 @@ cudaError_t launch_selftest_wait(WsHeader* hdr, dst_result_t* result, long long 
 cudaError_t launch_reduce_rows(const MainArgs& a, int value_type, int out_type, bool vector_ok, int sm_count,
                                cudaStream_t stream) {
     if (a.apply) {
-        if (value_type != DST_F32 || out_type != DST_F32) return cudaErrorInvalidValue;
-        return launch_typed<float, float, true>(a, vector_ok, sm_count, stream);
+        // value rows and dense_in of one type; weight and state fp32
+        if (value_type != out_type) return cudaErrorInvalidValue;
+        if (value_type == DST_F32) {
+            if (a.apply == kOptSgd) return launch_typed<float, float, kOptSgd>(a, vector_ok, sm_count, stream);
+            if (a.apply == kOptMomentum) return launch_typed<float, float, kOptMomentum>(a, vector_ok, sm_count, stream);
+            if (a.apply == kOptAdam) return launch_typed<float, float, kOptAdam>(a, vector_ok, sm_count, stream);
+        } else {
+            if (a.apply == kOptSgd) return launch_typed<__nv_bfloat16, __nv_bfloat16, kOptSgd>(a, vector_ok, sm_count, stream);
+            if (a.apply == kOptMomentum) return launch_typed<__nv_bfloat16, __nv_bfloat16, kOptMomentum>(a, vector_ok, sm_count, stream);
+            if (a.apply == kOptAdam) return launch_typed<__nv_bfloat16, __nv_bfloat16, kOptAdam>(a, vector_ok, sm_count, stream);
+        }
+        return cudaErrorInvalidValue;
     }
     if (value_type == DST_F32 && out_type == DST_F32) return launch_typed<float, float>(a, vector_ok, sm_count, stream);
     if (value_type == DST_F32 && out_type == DST_BF16) return launch_typed<float, __nv_bfloat16>(a, vector_ok, sm_count, stream);
