@@ -58,6 +58,15 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<unsigned*>(&t);
 }
 
+// The square root and the quotient of Adam's step, 32 of each per lane and output row: the IEEE-rounded ones
+// cost about twenty instructions apiece and made the step instruction-bound; these are good to two units in
+// the last place, a hundredth of what the step's own rounding allows for.
+__device__ __forceinline__ float fast_sqrt(float x) {
+    float r;
+    asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
 // VC consecutive elements at p (shared or global memory, generic address) -> fp32
 __device__ __forceinline__ void load_elems(const float* p, Acc<4>& a) {
     float4 t = *reinterpret_cast<const float4*>(p);
@@ -174,13 +183,16 @@ enum : int {
 constexpr int kTabCache = 64;       // slices whose table is copied into shared memory
 constexpr int kHeavyCache = 1024;   // heavy rows whose first chunk id is copied into shared memory
 constexpr int kNamedWords = 65536 / 32;   // the overlapped path is for vocabularies of at most 65536 rows
+template <bool OVERLAP>
 struct CtaTables {
     long long start[kTabCache];
     unsigned long long values[kTabCache];
     int chunk_base[kHeavyCache];
     int n_heavy;
     int state;                     // overlapped path: 0 tables not loaded, 1 a warp is loading them, 2 loaded
-    unsigned named[kNamedWords];   // overlapped path: bit v set when some valid entry names row v
+    unsigned named[OVERLAP ? kNamedWords : 1];   // overlapped path: bit v set when some valid entry names row v
+    // (only there: the other variants size their CTAs per SM by shared memory, and 8 KB more would cost the
+    // bf16 kernel its fourth CTA)
 };
 
 // A block of at most 32 units, one per lane.
@@ -214,7 +226,7 @@ struct WarpPipe {
     const unsigned bars;      // shared address of this warp's first mbarrier (one per slot)
     char* const ring_ptr;     // generic address of the first slot
     volatile int* const abort_flag;
-    CtaTables& tabs;          // this CTA's shared copies of the slice table and of the heavy rows' first chunk ids
+    CtaTables<OVERLAP>& tabs; // this CTA's shared copies of the slice table and of the heavy rows' first chunk ids
     HeavyInfo cur_heavy;      // the heavy row of the chunk item being processed
     int islot;                // slot the next issued unit goes to
     int cslot;                // slot of the next unit to consume
@@ -225,7 +237,7 @@ struct WarpPipe {
     Acc<VC> aux[K];           // kOptAdam: sqrt(vhat) + eps of the row being closed, between its v unit and its m unit
 
     __device__ WarpPipe(const MainArgs& args, unsigned ring_addr, unsigned bar_addr, char* ring_generic, volatile int* ab,
-                        CtaTables& t)
+                        CtaTables<OVERLAP>& t)
         : a(args), lane(lane_id()), ring(ring_addr), bars(bar_addr), ring_ptr(ring_generic), abort_flag(ab), tabs(t), islot(0),
           cslot(0), cphase(0u), issued_mask(0u), polled(0), ns(args.n_slots) {}
 
@@ -243,7 +255,7 @@ struct WarpPipe {
         for (int i = 0; i < VC; ++i) {
             g.x[i] = a.grad_scale * g.x[i];
             s.x[i] = fmaf(a.opt_b, s.x[i], (1.f - a.opt_b) * (g.x[i] * g.x[i]));
-            den.x[i] = sqrtf(s.x[i] * a.opt_bc2) + a.opt_eps;
+            den.x[i] = fast_sqrt(s.x[i] * a.opt_bc2) + a.opt_eps;
         }
     }
     // second state unit of kOptAdam: s holds m; leaves the new m in s and the bias-corrected step direction in g
@@ -251,7 +263,7 @@ struct WarpPipe {
 #pragma unroll
         for (int i = 0; i < VC; ++i) {
             s.x[i] = fmaf(a.opt_a, s.x[i], (1.f - a.opt_a) * g.x[i]);
-            g.x[i] = (s.x[i] * a.opt_bc1) / den.x[i];
+            g.x[i] = __fdividef(s.x[i] * a.opt_bc1, den.x[i]);
         }
     }
     // the weight unit: w holds the weight row; g what the state units left (kOptSgd: the raw sum)
@@ -903,7 +915,7 @@ __global__ void __launch_bounds__(kPipeThreads, (sizeof(VT) == 2 && OPT == kOptN
 k_reduce_rows(const __grid_constant__ MainArgs a) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ int s_abort;
-    __shared__ CtaTables tabs;
+    __shared__ CtaTables<OVERLAP> tabs;
     unsigned long long* bar_base = reinterpret_cast<unsigned long long*>(smem_raw);
     char* slot_base = reinterpret_cast<char*>(smem_raw) + kPipeHeaderReserve;
     const int warp = warp_id();
