@@ -131,6 +131,34 @@ int dst_densify_concat(const dst_slice_t* slices, int32_t R, int64_t d, int64_t 
                        void* unique_rows, int32_t* counts, dst_result_t* result);
 
 /*
+ * The whole "after" pipeline of the paper in one pass (Section 4, Fig. 3b: every rank converts its own
+ * IndexedSlices, then everything is reduced; Fig. 5 for the sizes): the gradients R ranks hold for the
+ * tied weight -- per rank one dense [vocab, d] tensor (the projection gradient, may be NULL) and any
+ * number of IndexedSlices (the embedding lookups) -- accumulated into one dense tensor,
+ *
+ *     out[v, c] = sum over ranks r of ( dense_r[v, c] + sum of rank r's value rows that name v )
+ *
+ * Every dense tensor and every value row is read once, on the way to its output row, and `out` is
+ * written once; no per-rank dense gradient and no running sum is ever materialised.  `ranks` is a
+ * HOST array of R descriptors (device pointers inside; `slices` a HOST array of n_slices entries),
+ * read during the call only.  At most 64 ranks may bring a dense tensor (DST_ERR_UNSUPPORTED beyond;
+ * dst_accumulate takes longer lists).  A row's value rows are summed first, in rank and slice order as
+ * dst_densify_concat would take the concatenation of all slices, then the dense rows in rank order.
+ * `out` may be one of the dense tensors.  Workspace: dst_workspace_bytes(all slice rows, all slices,
+ * d, vocab, opts).  Everything else as dst_densify_concat.
+ */
+typedef struct {
+    const void* dense;         /* [vocab, d] in opts->out_type, or NULL */
+    const dst_slice_t* slices; /* host array */
+    int32_t n_slices;
+    int32_t reserved;
+} dst_rank_grads_t;
+
+int dst_densify_batch(const dst_rank_grads_t* ranks, int32_t R, int64_t d, int64_t vocab, void* out,
+                      dst_stream_t stream, const dst_opts_t* opts, void* workspace, size_t workspace_bytes,
+                      void* unique_rows, int32_t* counts, dst_result_t* result);
+
+/*
  * dst_densify_concat fused with the step that follows accumulation in the training loop (Section 4:
  * the optimizer the accumulated gradient is handed to), for plain SGD on the tied weight:
  *
@@ -258,12 +286,13 @@ int dst_densify_concat_host(const dst_slice_t* slices, int32_t R, int64_t d, int
  * (dst_workspace_bytes(plan.n_slice_rows, plan.n_slices, d, vocab, opts) when plan.converts != 0).
  *
  * dst_accumulate enqueues the work on `stream`:
- *   - dense output  -> out_dense [vocab, d] in opts->out_type.  The dense gradients are added in fp32
- *     in the order given, eight tensors per pass (with more than eight the running sum passes
- *     through out_dense, in opts->out_type, between passes); a gradient that is out_dense itself is
- *     taken first, so that it is read before the first pass overwrites it.  Then the slices are
- *     densified onto that sum in one pass (dst_densify_concat with out_dense as its dense partner),
- *     so the value rows cross the memory bus once.
+ *   - dense output  -> out_dense [vocab, d] in opts->out_type, summed in fp32.  With IndexedSlices
+ *     among the gradients (or more than eight dense ones and a workspace) everything is accumulated
+ *     in one pass, as dst_densify_batch does: a row's value rows first, then the dense gradients in
+ *     the order given, except that a gradient that is out_dense itself is taken first; every tensor
+ *     crosses the memory bus once.  More than 64 dense gradients: the first ones are summed into
+ *     out_dense beforehand (eight per pass, the running sum in opts->out_type between passes).
+ *     Dense gradients only, at most eight or without a workspace: those passes alone.
  *     `result` (optional) is written only when slices were converted (plan.converts != 0).
  *   - slices output -> out_indices [out_rows], out_values [out_rows, d]: the concatenation.  Needs
  *     out_capacity_rows >= plan.out_rows, and value_type == out_type when a dense gradient is

@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     dst_bytes_report,
     dst_densify,
     dst_densify_apply,
+    dst_densify_batch,
     dst_densify_apply_sgd,
     dst_densify_concat,
     dst_densify_concat_host,

@@ -53,6 +53,11 @@ class _Optimizer(ctypes.Structure):
                 ("grad_scale", ctypes.c_float), ("state1", ctypes.c_void_p), ("state2", ctypes.c_void_p)]
 
 
+class _RankGrads(ctypes.Structure):
+    _fields_ = [("dense", ctypes.c_void_p), ("slices", ctypes.POINTER(_Slice)), ("n_slices", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
 class _Grad(ctypes.Structure):
     _fields_ = [("kind", ctypes.c_int32), ("reserved", ctypes.c_int32), ("indices", ctypes.c_void_p),
                 ("values", ctypes.c_void_p), ("n_rows", ctypes.c_int64)]
@@ -84,6 +89,8 @@ SYMBOLS = {
                                              ctypes.POINTER(_Opts), _vp, _sz, _vp, _vp, _vp]),
     "dst_densify_apply": (ctypes.c_int, [ctypes.POINTER(_Slice), _i32, _i64, _i64, _vp, _vp, ctypes.POINTER(_Optimizer), _vp,
                                          ctypes.POINTER(_Opts), _vp, _sz, _vp, _vp, _vp]),
+    "dst_densify_batch": (ctypes.c_int, [ctypes.POINTER(_RankGrads), _i32, _i64, _i64, _vp, _vp, ctypes.POINTER(_Opts),
+                                         _vp, _sz, _vp, _vp, _vp]),
     "dst_densify_static": (ctypes.c_int, [_vp, _vp, _i64, _i64, _i64, _vp, _vp, _vp, ctypes.POINTER(_Opts),
                                           _vp, _vp, _vp]),
     "dst_host_staging_bytes": (_sz, [_i64, _i64, _i64, ctypes.POINTER(_Opts)]),
@@ -278,6 +285,38 @@ def dst_densify_apply_sgd(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]], d
                                        _ptr(unique_rows), _ptr(counts), _ptr(result))
     if rc != 0:
         raise DstError(rc, "dst_densify_apply_sgd")
+
+
+def dst_densify_batch(ranks, d: int, vocab: int, out: torch.Tensor, workspace: torch.Tensor,
+                      unique_rows: Optional[torch.Tensor] = None, counts: Optional[torch.Tensor] = None,
+                      result: Optional[torch.Tensor] = None, stream=None, index_dtype: Optional[torch.dtype] = None,
+                      value_dtype: Optional[torch.dtype] = None) -> None:
+    """Enqueue ``dst_densify_batch`` (include/dst.h).  ``ranks``: a list of (dense or None, [(indices, values), ...])."""
+    lib = load_library()
+    R = len(ranks)
+    arr = (_RankGrads * max(R, 1))()
+    keep = []
+    for r, (dense, slices) in enumerate(ranks):
+        if dense is not None and (dense.dtype != out.dtype or dense.numel() != vocab * d or not dense.is_contiguous()):
+            raise ValueError("a rank's dense tensor must be contiguous [vocab, d] in out's dtype")
+        sl = (_Slice * max(len(slices), 1))()
+        for q, (idx, val) in enumerate(slices):
+            index_dtype = index_dtype or idx.dtype
+            value_dtype = value_dtype or val.dtype
+            if idx.dtype != index_dtype or val.dtype != value_dtype:
+                raise TypeError("all slices must share index and value dtypes")
+            _check_slice(idx, val, d, out.device)
+            sl[q].indices, sl[q].values, sl[q].n_rows = idx.data_ptr(), val.data_ptr(), idx.shape[0]
+        keep.append(sl)
+        arr[r].dense = dense.data_ptr() if dense is not None else None
+        arr[r].slices = ctypes.cast(sl, ctypes.POINTER(_Slice))
+        arr[r].n_slices = len(slices)
+    o = _opts(index_dtype or torch.int64, value_dtype or torch.float32, out.dtype)
+    with torch.cuda.device(out.device):
+        rc = lib.dst_densify_batch(arr, R, d, vocab, _ptr(out), _stream_handle(stream), ctypes.byref(o), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _ptr(unique_rows), _ptr(counts), _ptr(result))
+    if rc != 0:
+        raise DstError(rc, "dst_densify_batch")
 
 
 def dst_densify_apply(slices: Sequence[Tuple[torch.Tensor, torch.Tensor]], d: int, vocab: int,

@@ -37,16 +37,22 @@ static int sm_count() {
     return n;
 }
 
-static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
-                        void* out, cudaStream_t stream, const dst_opts_t* opts, void* workspace,
+// `dense`: the n_dense dense partners (n_dense <= kMaxDensePartners, no null among them), added after the value
+// rows in the order given.
+static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* const* dense,
+                        int n_dense, void* out, cudaStream_t stream, const dst_opts_t* opts, void* workspace,
                         size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result,
                         const dst_optimizer_t* optimizer = nullptr) {
     if (!opts_ok(opts)) return opts ? DST_ERR_UNSUPPORTED : DST_ERR_INVALID_ARG;
+    if (n_dense < 0 || n_dense > kMaxDensePartners || (n_dense > 0 && !dense)) return DST_ERR_INVALID_ARG;
+    for (int p = 0; p < n_dense; ++p) if (!dense[p]) return DST_ERR_INVALID_ARG;
+    const void* dense_in = n_dense > 0 ? dense[0] : nullptr;
     const bool apply = optimizer != nullptr;
     // with an optimizer `out` is the fp32 weight; value rows and dense_in share one type
     if (apply && opts->value_type != opts->out_type) return DST_ERR_UNSUPPORTED;
-    if (apply && out && (out == dense_in || out == optimizer->state1 || out == optimizer->state2))
-        return DST_ERR_INVALID_ARG;                                    // the weight is not its own gradient or state
+    if (apply && out && (out == optimizer->state1 || out == optimizer->state2))
+        return DST_ERR_INVALID_ARG;                                    // the weight is not its own state
+    for (int p = 0; apply && p < n_dense; ++p) if (dense[p] == out) return DST_ERR_INVALID_ARG;   // nor its own gradient
     if (apply) {
         const int k = optimizer->kind;
         if (k != DST_OPT_SGD && k != DST_OPT_MOMENTUM && k != DST_OPT_ADAM) return DST_ERR_INVALID_ARG;
@@ -89,7 +95,8 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     // the fast kernels need 16-byte aligned rows everywhere
     const size_t smallest = dtype_size(opts->value_type) < dtype_size(opts->out_type) ? dtype_size(opts->value_type)
                                                                                       : dtype_size(opts->out_type);
-    bool vector_ok = d % int64_t(16 / smallest) == 0 && aligned16(out) && aligned16(dense_in);
+    bool vector_ok = d % int64_t(16 / smallest) == 0 && aligned16(out);
+    for (int p = 0; p < n_dense; ++p) vector_ok = vector_ok && aligned16(dense[p]);
     if (apply) vector_ok = vector_ok && aligned16(optimizer->state1) && aligned16(optimizer->state2);
     for (int r = 0; r < R && vector_ok; ++r)
         if (slices[r].n_rows > 0 && !aligned16(slices[r].values)) vector_ok = false;
@@ -118,7 +125,8 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         fp.nodecnt_words = int((L.off_batches - L.off_nodecnt) / 4);
         compact = true;
         // (plain SGD without a dense partner leaves the rows nobody names alone; momentum and Adam move every row)
-        overlap = apply ? (dense_in != nullptr || optimizer->kind != DST_OPT_SGD) : out != dense_in;
+        // (several dense partners: every row is at least their sum)
+        overlap = apply ? (n_dense > 0 || optimizer->kind != DST_OPT_SGD) : (n_dense > 1 || out != dense_in);
         fp.urec = reinterpret_cast<unsigned*>(ws + L.off_urow);
         fp.bitmap = reinterpret_cast<unsigned*>(ws + L.off_bitmap);
         fp.bitmap_words = L.bitmap_words;
@@ -171,6 +179,8 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     MainArgs a;
     a.hdr = hdr; a.offsets = offsets; a.perm = perm; a.tab = tab; a.heavy = heavy;
     a.batches = batches; a.node_cnt = nodecnt; a.partials = partials; a.dense_in = dense_in; a.out = out;
+    a.n_dense = n_dense;
+    for (int p = 1; p < kMaxDensePartners; ++p) a.dense_more[p - 1] = p < n_dense ? dense[p] : nullptr;
     a.result = result; a.d = d; a.vocab = int(vocab); a.n_total = int(n_total); a.R = R; a.chunk = L.chunk;
     a.chunk_max = int(L.chunk_max); a.upper_max = int(L.upper_max);
     a.W = a.ncb = a.slot_bytes = a.n_slots = 0;   // set by the launcher
@@ -268,15 +278,15 @@ int dst_densify(const void* indices, const void* values, int64_t n_rows, int64_t
                 const void* dense_in, void* out, dst_stream_t stream, const dst_opts_t* opts, void* workspace,
                 size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
     dst_slice_t s{indices, values, n_rows};
-    return densify_impl(&s, 1, d, vocab, dense_in, out, stream, opts, workspace, workspace_bytes, unique_rows,
-                        counts, result);
+    return densify_impl(&s, 1, d, vocab, &dense_in, dense_in ? 1 : 0, out, stream, opts, workspace, workspace_bytes,
+                        unique_rows, counts, result);
 }
 
 int dst_densify_concat(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
                        void* out, dst_stream_t stream, const dst_opts_t* opts, void* workspace,
                        size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
-    return densify_impl(slices, R, d, vocab, dense_in, out, stream, opts, workspace, workspace_bytes, unique_rows,
-                        counts, result);
+    return densify_impl(slices, R, d, vocab, &dense_in, dense_in ? 1 : 0, out, stream, opts, workspace, workspace_bytes,
+                        unique_rows, counts, result);
 }
 
 int dst_densify_apply_sgd(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
@@ -285,16 +295,16 @@ int dst_densify_apply_sgd(const dst_slice_t* slices, int32_t R, int64_t d, int64
     if (opts_ok(opts) && (opts->value_type != DST_F32 || opts->out_type != DST_F32)) return DST_ERR_UNSUPPORTED;
     dst_optimizer_t sgd{};
     sgd.kind = DST_OPT_SGD; sgd.lr = lr; sgd.grad_scale = 1.f;
-    return densify_impl(slices, R, d, vocab, dense_in, weight, stream, opts, workspace, workspace_bytes, unique_rows,
-                        counts, result, &sgd);
+    return densify_impl(slices, R, d, vocab, &dense_in, dense_in ? 1 : 0, weight, stream, opts, workspace, workspace_bytes,
+                        unique_rows, counts, result, &sgd);
 }
 
 int dst_densify_apply(const dst_slice_t* slices, int32_t R, int64_t d, int64_t vocab, const void* dense_in,
                       void* weight, const dst_optimizer_t* optimizer, dst_stream_t stream, const dst_opts_t* opts,
                       void* workspace, size_t workspace_bytes, void* unique_rows, int32_t* counts, dst_result_t* result) {
     if (!optimizer) return DST_ERR_INVALID_ARG;
-    return densify_impl(slices, R, d, vocab, dense_in, weight, stream, opts, workspace, workspace_bytes, unique_rows,
-                        counts, result, optimizer);
+    return densify_impl(slices, R, d, vocab, &dense_in, dense_in ? 1 : 0, weight, stream, opts, workspace, workspace_bytes,
+                        unique_rows, counts, result, optimizer);
 }
 
 int dst_densify_static(const void* indices, const void* values, int64_t n_rows, int64_t d, int64_t vocab,
@@ -310,7 +320,7 @@ int dst_densify_static(const void* indices, const void* values, int64_t n_rows, 
     void* ws = nullptr;
     if (static_workspace(&ws) != cudaSuccess) return DST_ERR_CUDA;
     dst_slice_t s{indices, values, n_rows};
-    return densify_impl(&s, 1, d, vocab, dense_in, out, stream, opts, ws, size_t(DST_STATIC_WORKSPACE_BYTES),
+    return densify_impl(&s, 1, d, vocab, &dense_in, dense_in ? 1 : 0, out, stream, opts, ws, size_t(DST_STATIC_WORKSPACE_BYTES),
                         unique_rows, counts, result);
 }
 
@@ -364,7 +374,8 @@ int dst_densify_concat_host(const dst_slice_t* slices, int32_t R, int64_t d, int
         cudaMemcpyAsync(d_out, host_dense_in, out_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return DST_ERR_CUDA;
     dst_slice_t s{d_idx, d_val, n_total};
-    int rc = densify_impl(&s, 1, d, vocab, host_dense_in ? d_out : nullptr, d_out, stream, opts, workspace,
+    const void* partner = d_out;
+    int rc = densify_impl(&s, 1, d, vocab, &partner, host_dense_in ? 1 : 0, d_out, stream, opts, workspace,
                           workspace_bytes, nullptr, nullptr, d_res);
     if (rc != DST_OK) return rc;
     if (cudaMemcpyAsync(host_out, d_out, out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return DST_ERR_CUDA;
@@ -472,48 +483,57 @@ int dst_accumulate(const dst_grad_t* grads, int32_t n, int64_t d, int64_t vocab,
         return DST_OK;
     }
 
-    // dense output: the dense gradients first, left to right, then the slices on top in one pass
+    // dense output.  The dense gradients in the order given, except that one that is out_dense itself goes first
+    // (it must be read before anything lands in out_dense).
     if (!out_dense) return DST_ERR_INVALID_ARG;
     const long long n_elems = (long long)vocab * d;
-    const void* partner = nullptr;          // what the slices are added to
-    if (p.n_dense == 1 && p.n_slices > 0) {
-        for (int i = 0; i < n; ++i) if (grads[i].kind == DST_GRAD_DENSE) partner = grads[i].values;
-    } else if (p.n_dense >= 1) {
-        // The dense gradients in the order given, except that a gradient out_dense aliases goes first: the
-        // running sum lands in out_dense after every kSumFanIn tensors, which must not happen before that
-        // gradient has been read.
+    std::unique_ptr<const void*[]> list(new (std::nothrow) const void*[p.n_dense + 1]);
+    if (!list) return DST_ERR_INVALID_ARG;
+    int n_list = 0, n_aliased = 0;
+    for (int round = 0; round < 2; ++round)
+        for (int i = 0; i < n; ++i)
+            if (grads[i].kind == DST_GRAD_DENSE && (grads[i].values == out_dense) == (round == 0)) {
+                list[n_list++] = grads[i].values;
+                n_aliased += round == 0;
+            }
+    if (n_aliased > kSumFanIn) return DST_ERR_INVALID_ARG;
+
+    // out_dense = list[0] + ... + list[count - 1], kSumFanIn tensors per pass, the running sum carried in out_dense
+    auto sum_passes = [&](int count) -> int {
         SumParams sp{};
         sp.out = out_dense; sp.n_elems = n_elems; sp.vector_ok = aligned16(out_dense);
         bool first = true;
-        int n_aliased = 0;
-        for (int i = 0; i < n; ++i)
-            if (grads[i].kind == DST_GRAD_DENSE && grads[i].values == out_dense) ++n_aliased;
-        if (n_aliased > kSumFanIn) return DST_ERR_INVALID_ARG;       // they would not all be read before the first write
-        for (int pos = n_aliased ? -n : 0; pos < n; ++pos) {
-            // first round (pos < 0): the gradients that are out_dense itself; second round: all others
-            const int i = pos < 0 ? pos + n : pos;
-            if (grads[i].kind != DST_GRAD_DENSE || (grads[i].values == out_dense) != (pos < 0)) continue;
-            sp.src[sp.k++] = grads[i].values;
-            sp.vector_ok = sp.vector_ok && aligned16(grads[i].values);
-            if (sp.k == kSumFanIn) {
-                if (launch_sum_dense(sp, opts->out_type, sm_count(), stream) != cudaSuccess) return DST_ERR_CUDA;
-                ++g_launches;
+        for (int q = 0; q < count; ++q) {
+            sp.src[sp.k++] = list[q];
+            sp.vector_ok = sp.vector_ok && aligned16(list[q]);
+            if (sp.k == kSumFanIn || q == count - 1) {
+                const bool nothing = first && sp.k == 1 && sp.src[0] == out_dense;   // one tensor that already is the output
+                if (!nothing && !(!first && sp.k == 1)) {
+                    if (launch_sum_dense(sp, opts->out_type, sm_count(), stream) != cudaSuccess) return DST_ERR_CUDA;
+                    ++g_launches;
+                }
                 first = false;
-                sp.k = 0; sp.src[sp.k++] = out_dense; sp.vector_ok = aligned16(out_dense);   // carry on from the running sum
+                sp.k = 0; sp.src[sp.k++] = out_dense; sp.vector_ok = aligned16(out_dense);
             }
         }
-        if (first ? sp.k >= 1 : sp.k >= 2) {
-            if (sp.k == 1 && sp.src[0] == out_dense) {
-                // a single dense gradient that already is the output
-            } else {
-                if (launch_sum_dense(sp, opts->out_type, sm_count(), stream) != cudaSuccess) return DST_ERR_CUDA;
-                ++g_launches;
-            }
-        }
-        partner = out_dense;
+        return DST_OK;
+    };
+
+    const size_t ws_need = make_layout(p.n_slice_rows, p.n_slices, d, vocab, int(dtype_size(opts->value_type)),
+                                       int(dtype_size(opts->out_type))).total;
+    const bool have_ws = workspace && workspace_bytes >= ws_need && !(reinterpret_cast<uintptr_t>(workspace) & 255u);
+    if (p.n_slices == 0 && (n_list <= kSumFanIn || !have_ws)) return sum_passes(n_list);   // a plain sum of dense tensors
+
+    // One pass over everything (Fig. 3b of the paper, all ranks at once): every dense tensor and every value row
+    // is read once on the way to its output row.  More dense tensors than one pass takes: the first ones are
+    // summed into out_dense beforehand, which then stands for them.
+    int first_in_pass = 0;
+    if (n_list > kMaxDensePartners) {
+        first_in_pass = n_list - (kMaxDensePartners - 1);
+        const int rc2 = sum_passes(first_in_pass);
+        if (rc2 != DST_OK) return rc2;
+        list[--first_in_pass] = out_dense;
     }
-    if (p.n_slices == 0) return DST_OK;
-    // convert_to_tensor of every IndexedSlices gradient (Listing 1), fused with the sum
     dst_slice_t stack_slices[64];
     dst_slice_t* sl = stack_slices;
     std::unique_ptr<dst_slice_t[]> heap;
@@ -525,8 +545,33 @@ int dst_accumulate(const dst_grad_t* grads, int32_t n, int64_t d, int64_t vocab,
     int r = 0;
     for (int i = 0; i < n; ++i)
         if (grads[i].kind == DST_GRAD_SLICES) sl[r++] = dst_slice_t{grads[i].indices, grads[i].values, grads[i].n_rows};
-    return densify_impl(sl, p.n_slices, d, vocab, partner, out_dense, stream, opts, workspace, workspace_bytes,
-                        nullptr, nullptr, result);
+    return densify_impl(sl, p.n_slices, d, vocab, list.get() + first_in_pass, n_list - first_in_pass, out_dense, stream, opts,
+                        workspace, workspace_bytes, nullptr, nullptr, result);
+}
+
+int dst_densify_batch(const dst_rank_grads_t* ranks, int32_t R, int64_t d, int64_t vocab, void* out, dst_stream_t stream,
+                      const dst_opts_t* opts, void* workspace, size_t workspace_bytes, void* unique_rows,
+                      int32_t* counts, dst_result_t* result) {
+    if (R < 0 || (R > 0 && !ranks)) return DST_ERR_INVALID_ARG;
+    const void* dense[kMaxDensePartners];
+    int n_dense = 0;
+    int64_t n_sl = 0;
+    for (int r = 0; r < R; ++r) {
+        if (ranks[r].n_slices < 0 || (ranks[r].n_slices > 0 && !ranks[r].slices)) return DST_ERR_INVALID_ARG;
+        if (ranks[r].dense) {
+            if (n_dense == kMaxDensePartners) return DST_ERR_UNSUPPORTED;
+            dense[n_dense++] = ranks[r].dense;
+        }
+        n_sl += ranks[r].n_slices;
+    }
+    if (n_sl > (1 << 20)) return DST_ERR_UNSUPPORTED;
+    std::unique_ptr<dst_slice_t[]> sl(new (std::nothrow) dst_slice_t[n_sl > 0 ? n_sl : 1]);
+    if (!sl) return DST_ERR_INVALID_ARG;
+    int64_t k = 0;
+    for (int r = 0; r < R; ++r)
+        for (int q = 0; q < ranks[r].n_slices; ++q) sl[k++] = ranks[r].slices[q];
+    return densify_impl(sl.get(), int32_t(n_sl), d, vocab, dense, n_dense, out, stream, opts, workspace, workspace_bytes,
+                        unique_rows, counts, result);
 }
 
 int dst_selftest_wait_limit(int64_t limit_cycles, void* workspace, size_t workspace_bytes, dst_stream_t stream,

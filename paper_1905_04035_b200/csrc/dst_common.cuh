@@ -42,6 +42,7 @@ constexpr unsigned kValueMask = 0x3FFFFFFFu;
 constexpr int64_t kMaxRows = (int64_t(1) << 30) - 1;  // look-back words keep 30 bits of count
 constexpr int64_t kMaxVocab = int64_t(1) << 30;
 constexpr int kSpinLimit = 1 << 20;
+constexpr int kMaxDensePartners = 64;       // dense tensors one densify pass adds (their pointers travel as kernel parameters)
 
 // ---- workspace --------------------------------------------------------------
 struct WsHeader {          // zeroed at the start of every call
@@ -122,10 +123,12 @@ struct MainArgs {
                            // (and perm[] holds 16-bit positions)
     unsigned* node_cnt;
     float* partials;
-    const void* dense_in;
+    const void* dense_in;   // the first dense partner (nullptr: none)
     void* out;
     dst_result_t* result;
     long long d;
+    int n_dense;            // dense partners in all: dense_in, then dense_more[0 .. n_dense - 2]
+    const void* dense_more[kMaxDensePartners - 1];
     int vocab;
     int n_total;     // rows in all slices (capacity of perm)
     int R;

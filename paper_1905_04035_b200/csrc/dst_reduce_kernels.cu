@@ -177,7 +177,8 @@ enum : int {
     kUnitChunkEnd = 8,   // last entry of chunk y: store the partial row, climb the tree
     kUnitPoll = 16,      // (copy items) ask now whether the index cluster has finished; the answer is looked at after the item
     kUnitState1 = 32,    // optimizer step: the slot holds the row of state1 (momentum buffer / Adam's m) of output row y
-    kUnitState2 = 64     // optimizer step: ... of state2 (Adam's v)
+    kUnitState2 = 64,    // optimizer step: ... of state2 (Adam's v)
+    kUnitAddDense = 128  // slot holds a row of a dense partner (dense_in's type): add it
 };
 
 constexpr int kTabCache = 64;       // slices whose table is copied into shared memory
@@ -273,17 +274,21 @@ struct WarpPipe {
     }
     // The units that close an output row, in ring order: its dense_in row (OPT: one more row to add), then,
     // with an optimizer, Adam's v row, the m / momentum row and last the weight row.
+    // There may be several dense partners (one per rank of the paper's Fig. 3b: every rank's projection gradient);
+    // each one's row of an output row is read once, on the way to that output row.
     __device__ __forceinline__ int n_closing() const {
-        if constexpr (!APPLY) return 1;
-        return (a.dense_in ? 1 : 0) + (OPT == kOptAdam ? 2 : (OPT == kOptMomentum ? 1 : 0)) + 1;
+        if constexpr (!APPLY) return a.n_dense > 1 ? a.n_dense : 1;
+        return a.n_dense + (OPT == kOptAdam ? 2 : (OPT == kOptMomentum ? 1 : 0)) + 1;
+    }
+    __device__ __forceinline__ const OT* dense_row_of(int which, long long at) const {
+        return static_cast<const OT*>(which == 0 ? a.dense_in : a.dense_more[which - 1]) + at;
     }
     __device__ __forceinline__ void closing_unit(UnitBlock& b, int c, long long at, long long wcols, bool named) const {
+        const unsigned dbytes = (unsigned)(wcols * (long long)sizeof(OT));
         if constexpr (APPLY) {
             const unsigned fbytes = (unsigned)(wcols * 4);
-            if (a.dense_in) {
-                if (c == 0) { b.src = static_cast<const OT*>(a.dense_in) + at; b.bytes = (unsigned)(wcols * (long long)sizeof(OT)); b.kind = kUnitAdd; return; }
-                --c;
-            }
+            if (c < a.n_dense) { b.src = dense_row_of(c, at); b.bytes = dbytes; b.kind = kUnitAddDense; return; }
+            c -= a.n_dense;
             if constexpr (OPT == kOptAdam) {
                 if (c == 0) { b.src = static_cast<const float*>(a.state2) + at; b.bytes = fbytes; b.kind = kUnitState2; return; }
                 --c;
@@ -293,9 +298,12 @@ struct WarpPipe {
                 --c;
             }
             b.src = static_cast<const float*>(a.out) + at; b.bytes = fbytes; b.kind = kUnitFinal;
+        } else if (c + 1 < a.n_dense) {
+            b.src = dense_row_of(c, at); b.bytes = dbytes; b.kind = kUnitAddDense;
         } else {
-            b.kind = kUnitFinal | (named ? 0 : kUnitCopy);
-            if (a.dense_in) { b.src = static_cast<const OT*>(a.dense_in) + at; b.bytes = (unsigned)(wcols * (long long)sizeof(OT)); }
+            // the last (or only) partner closes the row; a row nobody names with one partner is its copy, bit for bit
+            b.kind = kUnitFinal | ((named || a.n_dense > 1) ? 0 : kUnitCopy);
+            if (a.n_dense > 0) { b.src = dense_row_of(a.n_dense - 1, at); b.bytes = dbytes; }
         }
     }
     __device__ __forceinline__ float* state_row(int which, int y, long long cb) const {
@@ -346,12 +354,16 @@ struct WarpPipe {
     // flight, and the sum costs about one trip to memory however busy the memory system is.
     // bf16 value rows (slots half as wide as a partial row): direct loads, half of the column
     // groups at a time to save registers.
-    // `last_row`, when given, is one more fp32 row added after the children (the dense row at the root).
+    // `n_extra` more fp32 rows are added after the children: the rows at element offset `extra_at` of the dense
+    // partners (at the root of a heavy row).
     __device__ __forceinline__ bool sum_children(Acc<VC> (&acc)[K], int first_slot, int n_children, long long cb, int wcols,
-                                                 const float* last_row) {
+                                                 int n_extra, long long extra_at) {
         if constexpr (sizeof(VT) == 4) {
-            const int n = n_children + (last_row ? 1 : 0);
-            auto source = [&](int c) { return c < n_children ? partial_row(first_slot + c) + cb : last_row; };
+            const int n = n_children + n_extra;
+            auto source = [&](int c) {
+                return c < n_children ? static_cast<const float*>(partial_row(first_slot + c) + cb)
+                                      : reinterpret_cast<const float*>(dense_row_of(c - n_children, extra_at));
+            };
             // the partial rows were written with ordinary stores; the copy engine reads them
             asm volatile("fence.proxy.async;" ::: "memory");
 #pragma unroll
@@ -468,11 +480,9 @@ struct WarpPipe {
             const bool root = n_parent == 1;
             // fp32 rows in, fp32 dense rows: the root's dense row rides the ring behind the children
             constexpr bool kDenseInRing = sizeof(VT) == 4 && sizeof(OT) == 4;
-            const float* dense_row = nullptr;
-            if constexpr (kDenseInRing)
-                if (root && a.dense_in)
-                    dense_row = static_cast<const float*>(a.dense_in) + (long long)hi.row * a.d + cb;
-            if (!sum_children(acc, child_first + parent * kFanIn, n_children, cb, wcols, dense_row)) return false;
+            const long long row_at = (long long)hi.row * a.d + cb;
+            const int in_ring = (kDenseInRing && root) ? a.n_dense : 0;
+            if (!sum_children(acc, child_first + parent * kFanIn, n_children, cb, wcols, in_ring, row_at)) return false;
             if (root) {
                 // The output may be the dense input itself, so the compiler keeps loads and stores in
                 // program order: read the whole dense row first, then store, or every column group
@@ -481,8 +491,8 @@ struct WarpPipe {
                     // weight and state rows straight from memory (heavy rows are few): all loads of a step first
                     float* wrow = static_cast<float*>(a.out) + (long long)hi.row * a.d + cb;
                     if constexpr (!kDenseInRing) {
-                        if (a.dense_in) {
-                            const OT* drow = static_cast<const OT*>(a.dense_in) + (long long)hi.row * a.d + cb;
+                        for (int p = 0; p < a.n_dense; ++p) {
+                            const OT* drow = dense_row_of(p, row_at);
                             Acc<VC> dn[K];
 #pragma unroll
                             for (int k = 0; k < K; ++k) { zero(dn[k]); if (col(k) < wcols) load_elems(drow + col(k), dn[k]); }
@@ -522,22 +532,28 @@ struct WarpPipe {
                     }
                     return true;
                 }
-                const OT* din = kDenseInRing ? nullptr : static_cast<const OT*>(a.dense_in);
-                OT* out = static_cast<OT*>(a.out) + (long long)hi.row * a.d + cb;
+                // The output may be a dense partner itself, so the compiler keeps loads and stores in program
+                // order: read a whole dense row first, then store, or every column group pays its own trip.
+                OT* out = static_cast<OT*>(a.out) + row_at;
                 constexpr int KH = (sizeof(VT) == 2 && K >= 4) ? K / 2 : K;
+                const int direct = kDenseInRing ? 0 : a.n_dense;       // partners not yet added
 #pragma unroll
                 for (int h0 = 0; h0 < K; h0 += KH) {
-                    Acc<VC> dn[KH];
+                    for (int p = 0; p < direct; ++p) {
+                        const OT* drow = dense_row_of(p, row_at);
+                        Acc<VC> dn[KH];
 #pragma unroll
-                    for (int k = 0; k < KH; ++k) {
-                        const int c = col(h0 + k);
-                        zero(dn[k]);
-                        if (din && c < wcols) load_elems(din + (long long)hi.row * a.d + cb + c, dn[k]);
+                        for (int k = 0; k < KH; ++k) {
+                            const int c = col(h0 + k);
+                            zero(dn[k]);
+                            if (c < wcols) load_elems(drow + c, dn[k]);
+                        }
+#pragma unroll
+                        for (int k = 0; k < KH; ++k) add(acc[h0 + k], dn[k]);
                     }
 #pragma unroll
                     for (int k = 0; k < KH; ++k) {
                         const int c = col(h0 + k);
-                        add(acc[h0 + k], dn[k]);
                         if (c < wcols) store_out(out + c, acc[h0 + k]);
                     }
                 }
@@ -589,6 +605,17 @@ struct WarpPipe {
 #pragma unroll
                 for (int k = 0; k < K; ++k) add(acc[k], v[k]);
             }
+            if (kind & kUnitAddDense) {
+                Acc<VC> v[K];
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    const int c = col(k);
+                    zero(v[k]);
+                    if (c < wcols) load_elems(reinterpret_cast<const OT*>(sp) + c, v[k]);
+                }
+#pragma unroll
+                for (int k = 0; k < K; ++k) add(acc[k], v[k]);
+            }
             if constexpr (OPT == kOptMomentum || OPT == kOptAdam) {
                 if (kind & (kUnitState1 | kUnitState2)) {
                     // the slot holds a row of optimizer state: update it, keep what the next closing unit needs
@@ -619,7 +646,7 @@ struct WarpPipe {
                 for (int k = 0; k < K; ++k) {
                     const int c = col(k);
                     zero(dn[k]);
-                    if ((APPLY || a.dense_in) && c < wcols) load_elems(reinterpret_cast<const WT*>(sp) + c, dn[k]);
+                    if ((APPLY || a.n_dense > 0) && c < wcols) load_elems(reinterpret_cast<const WT*>(sp) + c, dn[k]);
                 }
 #pragma unroll
                 for (int k = 0; k < K; ++k) {
@@ -998,13 +1025,14 @@ k_reduce_rows_scalar(const MainArgs a) {
         const int v = (int)(e / a.d);
         const long long c = e - (long long)v * a.d;
         const int beg = max(a.offsets[v], 0), end = min(a.offsets[v + 1], a.n_total);
-        if (beg >= end && !a.apply) { static_cast<OT*>(a.out)[e] = din ? din[e] : OT(0.f); continue; }
+        if (beg >= end && !a.apply && a.n_dense <= 1) { static_cast<OT*>(a.out)[e] = din ? din[e] : OT(0.f); continue; }
         float acc = 0.f;
         for (int j = beg; j < end; ++j) {
             unsigned p = a.perm[j];
             if (p < (unsigned)a.n_total) acc += (float)resolve_row<VT>(a, p)[c];
         }
         if (din) acc += (float)din[e];
+        for (int q = 1; q < a.n_dense; ++q) acc += (float)static_cast<const OT*>(a.dense_more[q - 1])[e];
         if (!a.apply) { static_cast<OT*>(a.out)[e] = OT(acc); continue; }
         float* w = static_cast<float*>(a.out) + e;
         float g = a.grad_scale * acc;
