@@ -406,6 +406,71 @@ def time_accumulate(device, steps: int, warmup: int, seed: int):
     return rows
 
 
+def time_ranks(device, R: int, steps: int, warmup: int, seed: int):
+    """R ranks' gradients of the tied weight (per rank the dense projection gradient and two lookups of 5,000 rows,
+    the paper's 64-process case) accumulated three ways: in one pass (dst_densify_batch), in two (the dense
+    tensors summed first, the slices densified onto the sum), and as the gathered form of Algorithm 1 (everything
+    concatenated as IndexedSlices, then densified).  Bytes: what each way has to move at least."""
+    import torch
+    import paper_1905_04035_b200 as dst
+    peak, _ = measured_peak()
+    vocab, d, n_lookup = 33708, 1024, 5000
+    g = torch.Generator(device=device); g.manual_seed(seed)
+    p = 1.0 / torch.arange(1, vocab + 1, dtype=torch.float64) ** 1.1
+    cdf = torch.cumsum(p / p.sum(), 0).to(device)
+    ranks = []
+    for r in range(R):
+        dense = torch.randn(vocab, d, device=device, generator=g) * 0.02
+        sl = []
+        for _ in range(2):
+            idx = torch.searchsorted(cdf, torch.rand(n_lookup, device=device, generator=g, dtype=torch.float64)).clamp_(max=vocab - 1)
+            sl.append((idx, torch.randn(n_lookup, d, device=device, generator=g) * 0.02))
+        ranks.append((dense, sl))
+    n = 2 * n_lookup * R
+    out = torch.empty(vocab, d, device=device)
+    ws = torch.empty(dst.dst_workspace_bytes(n, 2 * R, d, vocab), dtype=torch.uint8, device=device)
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+    dense_b, value_b = vocab * d * 4, n * d * 4
+    all_slices = [s for _, sl in ranks for s in sl]
+    denses = [dn for dn, _ in ranks]
+    g_idx = torch.empty(R * vocab + n, dtype=torch.int64, device=device)
+    g_val = torch.empty(R * vocab + n, d, device=device)
+    ws_g = torch.empty(dst.dst_workspace_bytes(R * vocab + n, 1, d, vocab), dtype=torch.uint8, device=device)
+
+    def one_pass():
+        dst.dst_densify_batch(ranks, d, vocab, out, ws)
+
+    def two_pass():
+        dst.dst_accumulate(denses, d, vocab, dst.DST_ACC_PROPOSED, out_dense=out)          # no workspace: the sum passes
+        dst.dst_densify_concat(all_slices, d, vocab, out, out, ws)
+
+    def gathered():
+        dst.dst_accumulate(denses + all_slices, d, vocab, dst.DST_ACC_STOCK, out_indices=g_idx, out_values=g_val)
+        dst.dst_densify(g_idx, g_val, d, vocab, None, out, ws_g)
+
+    gather_b = (R * vocab + n) * (d * 4 + 8)
+    rows = []
+    for name, fn, nbytes in (("one pass (dst_densify_batch)", one_pass, R * dense_b + value_b + dense_b),
+                             ("two passes (sum of dense tensors, then densify onto it)", two_pass,
+                              R * dense_b + value_b + dense_b + 2 * dense_b * ((R + 6) // 7)),
+                             ("gathered form (Algorithm 1), then densified", gathered, 3 * gather_b + dense_b)):
+        for _ in range(warmup):
+            flush.zero_(); fn()
+        ev = []
+        for _ in range(steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            ev.append((a, b))
+        torch.cuda.synchronize()
+        ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+        rows.append({"way": name, "ms_per_step": ms, "bytes_moved_at_least": nbytes, "gbs": nbytes / ms / 1e6,
+                     "frac_of_hbm_peak": nbytes / ms / 1e6 / peak})
+    rep = dst.dst_bytes_report([2 * n_lookup] * R, d, vocab)       # per rank: both lookups
+    return {"R": R, "vocab": vocab, "d": d, "rows_per_lookup": n_lookup, "ways": rows,
+            "gathered_bytes": gather_b, "dense_bytes": dense_b, "bytes_report": rep}
+
+
 def time_e2e(w, device, steps: int, warmup: int):
     """Same metric through the host entry point: pinned host buffers, H2D and D2H inside the timed region."""
     import torch
@@ -629,8 +694,14 @@ def main():
                 targets[name] = {"ms_per_step": r["ms_per_step"], "frac": r["frac_of_hbm_peak"], "bar": TARGETS[name]}
 
     accumulate = None
+    ranks_rows = None
     if rank == 0 and world == 1 and not args.headline_only:
         accumulate = time_accumulate(device, min(args.steps, 50), args.warmup, args.seed)
+        torch.cuda.empty_cache()
+        ranks_rows = []
+        for R in (8, 64):
+            ranks_rows.append(time_ranks(device, R, min(args.steps, 10), 3, args.seed))
+            torch.cuda.empty_cache()
 
     cpu = cpu_threads = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -667,7 +738,7 @@ def main():
             "e2e": e2e, "gpu_launches": head["launches"], "clocks": head["clocks"],
             "cpu_baseline": cpu, "cpu_baseline_threads": cpu_threads, "bytes_report": rep,
             "parity": {"status": head["status"], "n_unique": head["n_unique"], "max_segment": head["max_segment"]},
-            "accumulate": accumulate, "all_configs": others,
+            "accumulate": accumulate, "ranks": ranks_rows, "all_configs": others,
         }
         print(json.dumps(line))
     if dist_ctx is not None:
