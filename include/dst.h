@@ -354,9 +354,13 @@ int dst_bytes_report(const int64_t* n_rows_per_slice, int32_t R, int64_t d, int6
  * row-reduction kernel (the kernel that moves the value, dense_in and out rows) on
  * the call's stream.  Pass NULL, NULL to switch it off (the default).
  * dst_kernel_launches: number of kernels this library has launched in this process.
+ * dst_profile_ranges: 1 switches on NVTX ranges on the calling host thread around a call and its
+ * phases (index work, row reduction), as a timeline tool shows them; 0 (the default) switches
+ * them off.  Process-wide; no environment variable is read.
  */
 void dst_profile_events(void* before, void* after);
 int64_t dst_kernel_launches(void);
+void dst_profile_ranges(int on);
 
 /*
  * Diagnostic of the library's bounded device-side waits (the paper has no counterpart: its

@@ -29,6 +29,7 @@ from .binding import (  # noqa: F401
     dst_host_staging_bytes,
     dst_kernel_launches,
     dst_profile_events,
+    dst_profile_ranges,
     dst_selftest_wait_limit,
     dst_status_string,
     dst_version,

@@ -99,6 +99,7 @@ SYMBOLS = {
     "dst_selftest_wait_limit": (ctypes.c_int, [_i64, _vp, _sz, _vp, _vp]),
     "dst_profile_events": (None, [_vp, _vp]),
     "dst_kernel_launches": (ctypes.c_int64, []),
+    "dst_profile_ranges": (None, [ctypes.c_int]),
     "dst_bytes_report": (ctypes.c_int, [ctypes.POINTER(_i64), _i32, _i64, _i64, ctypes.POINTER(_Opts),
                                         ctypes.POINTER(_BytesReport)]),
     "dst_accumulate_plan": (ctypes.c_int, [ctypes.POINTER(_Grad), _i32, _i64, _i64, _i32, ctypes.POINTER(_Opts),
@@ -177,6 +178,11 @@ def dst_profile_events(before=None, after=None) -> None:
 
 def dst_kernel_launches() -> int:
     return int(load_library().dst_kernel_launches())
+
+
+def dst_profile_ranges(on: bool) -> None:
+    """NVTX ranges around the phases of later calls (off by default)."""
+    load_library().dst_profile_ranges(1 if on else 0)
 
 
 def dst_selftest_wait_limit(limit_cycles: int, workspace: torch.Tensor, result: Optional[torch.Tensor] = None,

@@ -53,7 +53,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         if p.returncode != 0:
             raise RuntimeError("nvcc failed: %s" % " ".join(cmd))
     tmp = LIB_PATH + ".tmp.%d" % os.getpid()
-    subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
+    subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a", "-ldl"])
     os.replace(tmp, LIB_PATH)
     return LIB_PATH
 

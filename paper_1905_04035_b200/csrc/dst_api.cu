@@ -7,12 +7,22 @@
 #include <new>
 #include <mutex>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "dst_common.cuh"
 
 namespace dst {
 
 static thread_local cudaEvent_t t_ev_before = nullptr, t_ev_after = nullptr;
 static std::atomic<long long> g_launches{0};
+static std::atomic<int> g_ranges{0};    // NVTX ranges around the phases of a call: off unless dst_profile_ranges(1)
+
+// An NVTX range on the calling host thread for as long as the object lives (nothing when ranges are off).
+struct PhaseRange {
+    bool on;
+    explicit PhaseRange(const char* name) : on(g_ranges.load(std::memory_order_relaxed) != 0) { if (on) nvtxRangePushA(name); }
+    ~PhaseRange() { if (on) nvtxRangePop(); }
+};
 
 static size_t index_size(int t) { return t == DST_I64 ? 8 : 4; }
 static size_t dtype_size(int t) { return t == DST_F32 ? 4 : 2; }
@@ -108,8 +118,10 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     // rows only, and the row-reduction kernel, running beside the index cluster, gives the other rows their
     // dense_in row (or zeros, or the dense part of the SGD step) while the index work is under way.  In place
     // there is nothing to do for those rows.
+    PhaseRange call_range(apply ? "dst: densify + optimizer step" : "dst: densify");
     const bool small = n_total <= kFrontMaxRows && vocab <= 65536 && R <= kHistSlices && vector_ok && n_total <= vocab;
     if (small) {
+        PhaseRange index_range("dst: index cluster (validate, sort, tables)");
         FrontParams fp;
         memset(&fp.P, 0, sizeof fp.P);
         fp.P.n = R;
@@ -134,6 +146,7 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         ++g_launches;
         perm = pos[0];
     } else {
+        PhaseRange index_range("dst: index kernels (validate, radix passes, bounds, scan)");
         if (cudaMemsetAsync(ws, 0, L.zero_bytes, stream) != cudaSuccess) return DST_ERR_CUDA;
         // a1: validate and narrow, at most kHistSlices slices per launch
         int64_t start = 0;
@@ -203,6 +216,7 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         }
     }
     a.urec = reinterpret_cast<const unsigned*>(ws + L.off_urow);
+    PhaseRange reduce_range("dst: row reduction");
     if (t_ev_before && cudaEventRecord(t_ev_before, stream) != cudaSuccess) return DST_ERR_CUDA;
     if (launch_reduce_rows(a, opts->value_type, opts->out_type, vector_ok, sm_count(), stream) != cudaSuccess)
         return DST_ERR_CUDA;
@@ -254,6 +268,8 @@ void dst_profile_events(void* before, void* after) {
 }
 
 int64_t dst_kernel_launches(void) { return g_launches.load(); }
+
+void dst_profile_ranges(int on) { g_ranges.store(on ? 1 : 0); }
 
 const char* dst_status_string(int status) {
     switch (status) {

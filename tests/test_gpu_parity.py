@@ -393,3 +393,14 @@ def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
         dst.dst_selftest_wait_limit(0, ws, res)
     w = make_workload("tiny")                                         # and the next call is an ordinary one
     assert_parity(w, run_library(w))
+
+
+def test_nvtx_ranges_can_be_switched_on_and_change_nothing():
+    w = make_workload("tiny")
+    plain = run_library(w)
+    dst.dst_profile_ranges(True)
+    try:
+        ranged = run_library(w)
+    finally:
+        dst.dst_profile_ranges(False)
+    assert np.array_equal(raw_bits(plain.out), raw_bits(ranged.out))
