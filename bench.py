@@ -471,6 +471,33 @@ def time_ranks(device, R: int, steps: int, warmup: int, seed: int):
             "gathered_bytes": gather_b, "dense_bytes": dense_b, "bytes_report": rep}
 
 
+def time_reduce(w, device, steps: int, warmup: int, dist_ctx):
+    """The data-parallel step of Section 4 with its exchange: each rank densifies its own slices into the dense
+    tensor, which a sum all-reduce (NCCL) then combines.  Device time, max over ranks."""
+    import torch
+    from paper_1905_04035_b200.reduce import densify_then_reduce, exchange_bytes
+    from paper_1905_04035_b200.replicas import combine_over_ranks
+    prob = DeviceProblem(w, device, n_sets=1)
+    slices, dense, out = prob.sets[0]
+    step = lambda: densify_then_reduce(lambda: prob.eng(slices, dense, out), out, dist_ctx)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    dist_ctx.barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        step()
+    t1.record()
+    torch.cuda.synchronize()
+    agg = combine_over_ranks(t0.elapsed_time(t1) / steps, prob.balg, w.n_rows_total, dist_ctx, device)
+    world = dist_ctx.get_world_size()
+    esz = {"f32": 4, "bf16": 2}[w.out_dtype]
+    isz = {"i32": 4, "i64": 8}[w.index_dtype]
+    return {"ms_per_step": agg["ms_per_step"], "ranks": world, "collective": "all_reduce(sum) of [vocab, d]",
+            **exchange_bytes(w.vocab, w.d, esz, w.n_rows_total, isz, world)}
+
+
 def time_e2e(w, device, steps: int, warmup: int):
     """Same metric through the host entry point: pinned host buffers, H2D and D2H inside the timed region."""
     import torch
@@ -630,6 +657,9 @@ def main():
                     help="only the accumulation-strategy and fused-SGD calls (prints their rows, one GPU)")
     ap.add_argument("--scale", type=float, default=1.0,
                     help="shrink the rows per slice (profiling captures on a small case); 1.0 = the named configuration")
+    ap.add_argument("--reduce", action="store_true",
+                    help="with more than one rank: also time the step followed by a sum all-reduce of the dense output "
+                         "(a separate row; the headline stays the independent replicas, with no collective)")
     ap.add_argument("--reference-rows", type=int, default=None,
                     help="rows of the workload the reference arm processes per step (default: all of them, unless the "
                          "run would then take more than about three minutes)")
@@ -676,6 +706,10 @@ def main():
         eagg = combine_over_ranks(head["e2e"]["ms_per_step"], head["algorithmic_bytes"], w.n_rows_total, dist_ctx, device)
         e2e = {"value": eagg["gbs"], "unit": "GB/s", "h2d_bytes_per_step": head["e2e"]["h2d"],
                "d2h_bytes_per_step": head["e2e"]["d2h"], "ms_per_step": eagg["ms_per_step"]}
+
+    reduce_row = None
+    if args.reduce and world > 1:
+        reduce_row = time_reduce(w, device, min(args.steps, 50), args.warmup, dist_ctx)
 
     others = []
     targets = {}
@@ -738,7 +772,7 @@ def main():
             "e2e": e2e, "gpu_launches": head["launches"], "clocks": head["clocks"],
             "cpu_baseline": cpu, "cpu_baseline_threads": cpu_threads, "bytes_report": rep,
             "parity": {"status": head["status"], "n_unique": head["n_unique"], "max_segment": head["max_segment"]},
-            "accumulate": accumulate, "ranks": ranks_rows, "all_configs": others,
+            "accumulate": accumulate, "ranks": ranks_rows, "reduce": reduce_row, "all_configs": others,
         }
         print(json.dumps(line))
     if dist_ctx is not None:
