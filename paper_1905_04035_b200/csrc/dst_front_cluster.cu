@@ -22,7 +22,7 @@
 // between lives in shared memory.  The header with the flags is cleared before the dependent launch is
 // released.
 //
-// The tables list the named rows only (by rank u among them: row number urow[u], first entry uoff[u]),
+// The tables list the named rows only (by rank u among them: urec[u] packs the row number and its first entry),
 // which is why this path is taken only when there are no more input rows than vocabulary rows.
 // Limits: n_total <= kFrontMaxRows (positions fit 16 bits), vocab <= 65536 (keys fit 16 bits),
 // R <= kHistSlices (the slice table travels as a kernel parameter).

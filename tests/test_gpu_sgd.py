@@ -1,5 +1,5 @@
 """``dst_densify_apply_sgd`` through the C ABI against ``oracle.apply_sgd``: every path the densify call
-has (one-cluster index path with the pre-filled output, general path, heavy rows with their combine tree,
+has (one-cluster index path running beside the copy of the untouched rows, general path, heavy rows with their combine tree,
 several slices, no dense partner, rows that are not 16-byte multiples, out-of-range indices)."""
 import numpy as np
 import pytest
