@@ -148,6 +148,12 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
     } else {
         PhaseRange index_range("dst: index kernels (validate, radix passes, bounds, scan)");
         if (cudaMemsetAsync(ws, 0, L.zero_bytes, stream) != cudaSuccess) return DST_ERR_CUDA;
+        // With a vocabulary small enough, the validation kernel counts the entries of every row itself; the
+        // scan then rides in the launch of the first radix pass and no pass over the sorted keys is needed.
+        const bool early_count = n_total > 0 && vocab <= kCountInPrepMaxVocab;
+        ScanParams sp{hdr, count, offsets, heavy, unique_rows, counts, result, batches,
+                      reinterpret_cast<int*>(ws + L.off_scandesc), int(vocab), int(L.vocab_pad), L.chunk, L.batch_units,
+                      opts->index_type == DST_I64 ? 1 : 0};
         // a1: validate and narrow, at most kHistSlices slices per launch
         int64_t start = 0;
         for (int first = 0; first < R; first += kHistSlices) {
@@ -164,29 +170,34 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
             }
             int grid_x = int((longest + kPrepTile - 1) / kPrepTile);
             if (grid_x < 1) grid_x = 1;   // still writes the slice table
-            if (launch_prep(P, grid_x, opts->index_type, hdr, digit, keys[0], tab, vocab, L.passes, stream) != cudaSuccess)
+            if (launch_prep(P, grid_x, opts->index_type, hdr, digit, keys[0], tab, vocab, L.passes,
+                            early_count ? count : nullptr, stream) != cudaSuccess)
                 return DST_ERR_CUDA;
             ++g_launches;
         }
         if (n_total > 0) {
             // a4: least significant digit first; keys/positions ping-pong between two buffers
             for (int p = 0; p < L.passes; ++p) {
-                if (launch_radix_pass(int(L.n_tiles), hdr, keys[p & 1], p == 0 ? nullptr : pos[p & 1], keys[(p + 1) & 1],
+                // (the sorted keys of the last pass are read by the run-length kernel only)
+                unsigned* keys_out = early_count && p == L.passes - 1 ? nullptr : keys[(p + 1) & 1];
+                if (launch_radix_pass(int(L.n_tiles), hdr, keys[p & 1], p == 0 ? nullptr : pos[p & 1], keys_out,
                                       pos[(p + 1) & 1], digit + p * 256, desc + size_t(p) * size_t(L.n_tiles) * 256, p,
-                                      int(n_total), stream) != cudaSuccess)
+                                      int(n_total), early_count && p == 0 ? &sp : nullptr, stream) != cudaSuccess)
                     return DST_ERR_CUDA;
                 ++g_launches;
             }
             // a2: run lengths of the sorted keys
-            if (launch_bounds(hdr, keys[L.passes & 1], count, int(n_total), int(vocab), stream) != cudaSuccess)
-                return DST_ERR_CUDA;
-            ++g_launches;
+            if (!early_count) {
+                if (launch_bounds(hdr, keys[L.passes & 1], count, int(n_total), int(vocab), stream) != cudaSuccess)
+                    return DST_ERR_CUDA;
+                ++g_launches;
+            }
         }
         // a3/a5/a6
-        ScanParams sp{hdr, count, offsets, heavy, unique_rows, counts, result, batches,
-                      reinterpret_cast<int*>(ws + L.off_scandesc), int(vocab), int(L.vocab_pad), L.chunk, L.batch_units};
-        if (launch_scan(opts->index_type, sp, stream) != cudaSuccess) return DST_ERR_CUDA;
-        ++g_launches;
+        if (!early_count) {
+            if (launch_scan(sp, stream) != cudaSuccess) return DST_ERR_CUDA;
+            ++g_launches;
+        }
     }
     // a7/a8
     MainArgs a;

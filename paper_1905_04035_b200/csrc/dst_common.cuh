@@ -13,14 +13,16 @@
 namespace dst {
 
 // ---- fixed shape parameters -------------------------------------------------
-constexpr int kSortThreads = 256;           // threads of the histogram and radix-pass kernels
-constexpr int kSortItems = 16;              // keys per thread of a radix pass
-constexpr int kTile = kSortThreads * kSortItems;  // 4096 keys per CTA
+constexpr int kRadixThreads = 512;          // threads of a radix-pass CTA (a multiple of 256, the number of digits; 256 threads: 1 % slower on the 64-slice case)
+constexpr int kRadixItems = 8;              // keys per thread of a radix pass
+constexpr int kTile = kRadixThreads * kRadixItems;  // 4096 keys per CTA
 constexpr int kClusterCtas = 8;             // the one-kernel index path for small inputs: CTAs per cluster,
 constexpr int kFrontThreads = 1024;         // threads per CTA,
 constexpr int kFrontMaxRows = 65535;        // largest input (positions are packed into 16 bits)
 constexpr int kPrepItems = 8;               // indices per thread of the validation kernel
-constexpr int kPrepTile = kSortThreads * kPrepItems;
+constexpr int kPrepThreads = 1024;
+constexpr int kPrepTile = kPrepThreads * kPrepItems;
+constexpr int kCountInPrepMaxVocab = 65536; // up to here a CTA of the validation kernel can hold a 16-bit counter per row in shared memory
 constexpr int kMaxPasses = 4;               // 8-bit digits, keys below 2^31
 constexpr int kFanIn = 8;                   // children per node of the heavy-row combine tree
 constexpr int kMaxBatchUnits = 31;          // a light work item holds rows worth at most this many units (+ one row)
@@ -32,7 +34,7 @@ constexpr int kPipeSlots = 6;               // ring slots per warp, at most
 constexpr int kPipeHeaderReserve = 1024;    // mbarriers in front of the slots
 constexpr int kMaxBlockCols = 1024;         // columns per column block (32 fp32 accumulators per lane)
 constexpr long long kWaitCycles = 1LL << 31; // SM clock cycles (about a second) before an mbarrier wait gives up
-constexpr int kScanThreads = 256;
+constexpr int kScanThreads = kRadixThreads;  // the scan tiles can ride in the launch of the first radix pass
 constexpr int kScanItems = 4;               // rows per thread in the scan kernel (16: 2 % slower on r64, 8: 0.5 %)
 constexpr int kScanTile = kScanThreads * kScanItems;
 constexpr int kSmCount = 148;               // B200; only used to pick the chunk length
@@ -244,12 +246,15 @@ struct ScanParams {
     int2* batches;
     int* scan_desc;
     int vocab, vocab_pad, chunk, batch_units;
+    int wide;              // unique_rows holds 64-bit integers
 };
+// count != nullptr: the kernel also counts the entries of every row (vocab <= kCountInPrepMaxVocab)
 cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeader* hdr, unsigned* digit_hist,
-                        unsigned* keys, SliceEntry* tab, long long vocab, int passes, cudaStream_t stream);
+                        unsigned* keys, SliceEntry* tab, long long vocab, int passes, unsigned* count, cudaStream_t stream);
+// out_keys == nullptr: the last pass, whose keys nobody reads; scan != nullptr: the scan tiles ride in this launch
 cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
                               unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
-                              int pass, int capacity, cudaStream_t stream);
+                              int pass, int capacity, const ScanParams* scan, cudaStream_t stream);
 struct FrontParams {
     HistParams P;
     WsHeader* hdr;
@@ -270,7 +275,7 @@ struct FrontParams {
 cudaError_t launch_front_cluster(int index_type, const FrontParams& p, cudaStream_t stream);
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
                           cudaStream_t stream);
-cudaError_t launch_scan(int index_type, const ScanParams& p, cudaStream_t stream);
+cudaError_t launch_scan(const ScanParams& p, cudaStream_t stream);
 // ---- accumulation dispatcher (Algorithms 1 and 2) ----
 constexpr int kSumFanIn = 8;                // dense tensors summed per launch
 struct SumParams {

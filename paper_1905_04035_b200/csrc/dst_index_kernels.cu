@@ -17,23 +17,33 @@
 namespace dst {
 
 // ---------------------------------------------------------------------------
-// a1: validate, narrow to 32-bit keys, per-pass digit histograms
+// a1: validate, narrow to 32-bit keys, per-pass digit histograms; a2 when the vocabulary is small
+// enough for one 16-bit counter per row in a CTA's shared memory: the CTA counts its own entries
+// there (a CTA sees at most kPrepTile < 65536 of them) and adds the rows it has met to count[].
+// The counts are then known before the sort, not after it, and the scan that turns them into the
+// row tables can run beside the radix passes.
 // ---------------------------------------------------------------------------
-template <typename IT>
-__global__ void __launch_bounds__(kSortThreads)
+template <typename IT, bool COUNT>
+__global__ void __launch_bounds__(kPrepThreads)
 k_prep(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, unsigned* __restrict__ digit_hist,
-       unsigned* __restrict__ keys, SliceEntry* __restrict__ tab, long long vocab, int passes) {
+       unsigned* __restrict__ keys, SliceEntry* __restrict__ tab, long long vocab, int passes,
+       unsigned* __restrict__ count, int count_words) {
     __shared__ unsigned dh[kMaxPasses * 256];
-    pdl_trigger();
-    pdl_wait();
-
+    extern __shared__ __align__(16) unsigned rows16[];   // COUNT: two 16-bit counters per word, count_words words (a multiple of 4)
     const SliceEntry& se = P.s[blockIdx.y];
-    if (blockIdx.x == 0 && threadIdx.x == 0) tab[P.first + blockIdx.y] = se;
     const long long n = se.n_rows;
     const long long t0 = (long long)blockIdx.x * kPrepTile;
+    // shared memory is this CTA's own: cleared before the wait on the kernels before this one
+    if (t0 < n) {
+        for (int s = threadIdx.x; s < kMaxPasses * 256; s += kPrepThreads) dh[s] = 0;
+        if (COUNT)
+            for (int s = threadIdx.x * 4; s < count_words; s += kPrepThreads * 4)
+                *reinterpret_cast<uint4*>(rows16 + s) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    pdl_trigger();
+    pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 0) tab[P.first + blockIdx.y] = se;
     if (t0 >= n) return;
-
-    for (int s = threadIdx.x; s < kMaxPasses * 256; s += kSortThreads) dh[s] = 0;
     __syncthreads();
 
     const IT* __restrict__ idx = static_cast<const IT*>(se.indices);
@@ -42,174 +52,50 @@ k_prep(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, unsigne
     long long vals[kPrepItems];          // every index of this thread first: one trip to memory, not kPrepItems
 #pragma unroll
     for (int k = 0; k < kPrepItems; ++k) {
-        const long long i = t0 + k * kSortThreads + threadIdx.x;
+        const long long i = t0 + k * kPrepThreads + threadIdx.x;
         vals[k] = -1;
         if (i < n) vals[k] = (long long)idx[i];
     }
 #pragma unroll
     for (int k = 0; k < kPrepItems; ++k) {
-        const long long i = t0 + k * kSortThreads + threadIdx.x;
+        const long long i = t0 + k * kPrepThreads + threadIdx.x;
         const bool in = i < n;
         const long long v = vals[k];
         const bool ok = in && v >= 0 && v < vocab;
         const unsigned key = ok ? (unsigned)v : kInvalidKey;
         if (in) keys[se.start + i] = key;
         bad += in && !ok;
-        if (ok)
+        // a warp whose 32 indices are all the same row (one very frequent row) adds once
+        const unsigned k0 = __shfl_sync(0xFFFFFFFFu, key, 0);
+        const bool same = __all_sync(0xFFFFFFFFu, ok && key == k0);
+        if (same) {
+            if (lane == 0) {
+                for (int p = 0; p < passes; ++p) atomicAdd(&dh[p * 256 + ((key >> (8 * p)) & 255u)], 32u);
+                if (COUNT) atomicAdd(&rows16[key >> 1], 32u << (16 * (key & 1u)));
+            }
+        } else if (ok) {
             for (int p = 0; p < passes; ++p) atomicAdd(&dh[p * 256 + ((key >> (8 * p)) & 255u)], 1u);
+            if (COUNT) atomicAdd(&rows16[key >> 1], 1u << (16 * (key & 1u)));
+        }
     }
     __syncthreads();
-    for (int s = threadIdx.x; s < passes * 256; s += kSortThreads) {
+    for (int s = threadIdx.x; s < passes * 256; s += kPrepThreads) {
         unsigned c = dh[s];
         if (c) atomicAdd(&digit_hist[s], c);
     }
+    if (COUNT) {
+        for (int s = threadIdx.x * 4; s < count_words; s += kPrepThreads * 4) {
+            const uint4 w = *reinterpret_cast<const uint4*>(rows16 + s);
+            const unsigned ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (ww[q] & 0xFFFFu) atomicAdd(&count[2 * (s + q)], ww[q] & 0xFFFFu);
+                if (ww[q] >> 16) atomicAdd(&count[2 * (s + q) + 1], ww[q] >> 16);
+            }
+        }
+    }
     for (int o = 16; o > 0; o >>= 1) bad += __shfl_down_sync(0xFFFFFFFFu, bad, o);
     if (lane == 0 && bad) atomicAdd(&hdr->n_bad, (unsigned long long)bad);
-}
-
-// ---------------------------------------------------------------------------
-// a4: one stable 8-bit radix pass (least significant digit first), single sweep
-// over the keys with a decoupled look-back for the cross-tile prefix
-// ---------------------------------------------------------------------------
-// Exclusive prefix of digit d's count over the tiles before `tile`.  Every tile publishes its own
-// count first ("aggregate"), then walks back over its predecessors, four at a time, until it meets
-// one that has published its inclusive prefix.  Tiles start in ticket order, so every predecessor
-// is running or done; the wait on a missing descriptor is bounded all the same.
-__device__ __forceinline__ unsigned lookback_exclusive(volatile unsigned* desc, int tile, int d, unsigned cnt,
-                                                       WsHeader* hdr) {
-    if (tile == 0) { desc[d] = kFlagPrefix | cnt; return 0; }
-    desc[(size_t)tile * 256 + d] = kFlagAggregate | cnt;
-    unsigned excl = 0;
-    bool ok = true, done = false;
-    for (int t = tile - 1; t >= 0 && ok && !done; t -= 4) {
-        unsigned v[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) v[q] = t - q >= 0 ? desc[(size_t)(t - q) * 256 + d] : 0x80000000u;   // past tile 0: an empty prefix
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            if (done || !ok) break;
-            unsigned w = v[q];
-            int spins = 0;
-            while ((w & kFlagMask) == 0) {
-                if (++spins > kSpinLimit) { ok = false; break; }
-                __nanosleep(20);
-                w = desc[(size_t)(t - q) * 256 + d];
-            }
-            if (!ok) break;
-            excl += w & kValueMask;
-            if ((w & kFlagMask) == kFlagPrefix) done = true;
-        }
-    }
-    if (!ok) { raise_status(hdr, DST_ERR_TIMEOUT); excl = 0; }
-    desc[(size_t)tile * 256 + d] = kFlagPrefix | ((excl + cnt) & kValueMask);
-    return excl;
-}
-
-__global__ void __launch_bounds__(kSortThreads)
-k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, const unsigned* __restrict__ in_pos,
-             unsigned* __restrict__ out_keys, unsigned* __restrict__ out_pos,
-             const unsigned* __restrict__ digit_hist, unsigned* desc, int pass, int capacity) {
-    constexpr int kWarps = kSortThreads / 32;
-    __shared__ unsigned wh[kWarps][256];
-    __shared__ unsigned bin_base[256];
-    __shared__ unsigned wsum[kWarps];
-    __shared__ unsigned s_tile;
-    pdl_trigger();
-    pdl_wait();
-    if (threadIdx.x == 0) s_tile = atomicAdd(&hdr->ticket[pass], 1u);   // tiles start in id order
-    // asked for now, needed later: these two trips to memory overlap the ticket's
-    const unsigned n_bad = pass == 0 ? 0u : (unsigned)hdr->n_bad;
-    const unsigned g = digit_hist[threadIdx.x];   // kSortThreads == 256 digits
-    for (int s = threadIdx.x; s < kWarps * 256; s += kSortThreads) (&wh[0][0])[s] = 0;
-    __syncthreads();
-    const int tile = (int)s_tile;
-    // pass 0 reads every input position (invalid rows carry kInvalidKey and drop out);
-    // later passes read the survivors
-    const int n_in = capacity - (int)n_bad;
-    const long long t0 = (long long)tile * kTile;
-    if (t0 >= n_in) return;
-
-    const int lane = lane_id(), warp = warp_id();
-    const int shift = 8 * pass;
-    const unsigned lt_mask = (1u << lane) - 1u;
-    unsigned key[kSortItems], pos[kSortItems], rank[kSortItems];
-#pragma unroll
-    for (int k = 0; k < kSortItems; ++k) {
-        long long e = t0 + warp * (32 * kSortItems) + k * 32 + lane;
-        key[k] = kInvalidKey; pos[k] = 0;
-        if (e < n_in) {
-            key[k] = in_keys[e];
-            pos[k] = in_pos ? in_pos[e] : (unsigned)e;
-        }
-    }
-    // stable rank inside the warp's consecutive keys
-#pragma unroll
-    for (int k = 0; k < kSortItems; ++k) {
-        const bool valid = key[k] != kInvalidKey;
-        unsigned dg = (key[k] >> shift) & 255u;
-        unsigned m = match_digit(dg, valid);
-        int leader = valid ? __ffs(m) - 1 : lane;
-        unsigned pre = 0;
-        if (valid && lane == leader) { pre = wh[warp][dg]; wh[warp][dg] = pre + __popc(m); }
-        pre = __shfl_sync(0xFFFFFFFFu, pre, leader);
-        rank[k] = pre + __popc(m & lt_mask);
-        __syncwarp();
-    }
-    __syncthreads();
-    // per digit: exclusive prefix over the warps of this tile, tile total
-    const int d = threadIdx.x;   // kSortThreads == 256 digits
-    unsigned cnt = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) { unsigned t = wh[w][d]; wh[w][d] = cnt; cnt += t; }
-    // where digit d starts globally: exclusive scan of this pass's digit histogram
-    unsigned ginc = g;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { unsigned t = __shfl_up_sync(0xFFFFFFFFu, ginc, o); if (lane >= o) ginc += t; }
-    if (lane == 31) wsum[warp] = ginc;
-    __syncthreads();
-    unsigned gbase = ginc - g;
-    for (int w = 0; w < warp; ++w) gbase += wsum[w];
-    unsigned excl = lookback_exclusive(desc, tile, d, cnt, hdr);
-    bin_base[d] = gbase + excl;
-    __syncthreads();
-#pragma unroll
-    for (int k = 0; k < kSortItems; ++k) {
-        if (key[k] != kInvalidKey) {
-            unsigned dg = (key[k] >> shift) & 255u;
-            unsigned q = bin_base[dg] + wh[warp][dg] + rank[k];
-            if (q < (unsigned)capacity) {
-                out_keys[q] = key[k];
-                out_pos[q] = pos[k];
-            } else {
-                raise_status(hdr, DST_ERR_TIMEOUT);   // only reachable after a failed look-back
-            }
-        }
-    }
-}
-
-// ---------------------------------------------------------------------------
-// a2: run lengths of the sorted keys.  The first entry of a run subtracts its position from
-// count[key], the last one adds its position + 1: two atomics per distinct row, never contended.
-// ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-k_bounds(const WsHeader* __restrict__ hdr, const unsigned* __restrict__ keys, unsigned* __restrict__ count,
-         int capacity, int vocab) {
-    pdl_trigger();
-    pdl_wait();
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= capacity) return;
-    // the three keys and the number of valid entries are asked for together: one trip to memory.
-    // (Entries past the valid ones hold whatever the buffer held; they are read, never used.)
-    const unsigned k = keys[i];
-    const unsigned before = i > 0 ? keys[i - 1] : 0u;
-    const unsigned after = i + 1 < capacity ? keys[i + 1] : 0u;
-    const int n = capacity - (int)hdr->n_bad;
-    if (i >= n) return;
-    if (k >= (unsigned)vocab) return;                    // only after a failed look-back
-    const unsigned prev = i > 0 ? before : ~k;
-    const unsigned next = i + 1 < n ? after : ~k;
-    if (prev != k) atomicSub(&count[k], (unsigned)i);
-    if (next != k) atomicAdd(&count[k], (unsigned)i + 1u);
 }
 
 // ---------------------------------------------------------------------------
@@ -231,6 +117,7 @@ struct ScanArgs {
     int2* batches;
     int* scan_desc;        // per tile: [0] flag (1 own sums, 2 inclusive prefix too), [2..7] own sums, [8..13] inclusive prefix
     int vocab, vocab_pad, chunk, batch_units, n_tiles;
+    int wide;              // unique_rows holds 64-bit integers
 };
 
 
@@ -266,19 +153,15 @@ __device__ __forceinline__ Scan6 block_exclusive_scan(Scan6 x, Scan6& total, int
     return ex;
 }
 
-template <typename IT>
-__global__ void __launch_bounds__(kScanThreads)
-k_scan(const ScanArgs s) {
+// One scan tile.  Called by every thread of a CTA of kScanThreads threads, after the wait on the kernels before.
+__device__ __forceinline__ void scan_tile(const ScanArgs& s) {
     __shared__ int sm[kScanThreads / 32][6];
     __shared__ int s_prefix[6];
     __shared__ int s_nearest;
     __shared__ int s_tile;
     __shared__ int s_fail;
     WsHeader* hdr = s.hdr;
-    pdl_trigger();
-    pdl_wait();
     const int chunk = s.chunk, B = s.batch_units, vocab = s.vocab;
-    IT* unique_rows = static_cast<IT*>(s.unique_rows);
     if (threadIdx.x == 0) {
         s_tile = (int)atomicAdd(&hdr->scan_ticket, 1u);   // tiles start in id order
         // after a failed look-back count[] is not to be trusted: leave every table empty
@@ -381,7 +264,10 @@ k_scan(const ScanArgs s) {
             const int v = e0 + q;
             o[q] = run.v[0];
             if (cc > 0) {
-                if (unique_rows) unique_rows[run.v[1]] = (IT)v;
+                if (s.unique_rows) {
+                    if (s.wide) static_cast<long long*>(s.unique_rows)[run.v[1]] = v;
+                    else static_cast<int*>(s.unique_rows)[run.v[1]] = v;
+                }
                 if (s.counts_out) s.counts_out[run.v[1]] = cc;
                 run.v[1] += 1;
             }
@@ -435,21 +321,232 @@ k_scan(const ScanArgs s) {
     }
 }
 
+__global__ void __launch_bounds__(kScanThreads)
+k_scan(const ScanArgs s) {
+    pdl_trigger();
+    pdl_wait();
+    scan_tile(s);
+}
+
+// ---------------------------------------------------------------------------
+// a4: one stable 8-bit radix pass (least significant digit first), single sweep
+// over the keys with a decoupled look-back for the cross-tile prefix
+// ---------------------------------------------------------------------------
+// Exclusive prefix of digit d's count over the tiles before `tile`.  Every tile publishes its own
+// count first ("aggregate"), then walks back over its predecessors, four at a time, until it meets
+// one that has published its inclusive prefix.  Tiles start in ticket order, so every predecessor
+// is running or done; the wait on a missing descriptor is bounded all the same.
+__device__ __forceinline__ void lookback_publish(volatile unsigned* desc, int tile, int d, unsigned cnt) {
+    desc[(size_t)tile * 256 + d] = (tile == 0 ? kFlagPrefix : kFlagAggregate) | cnt;
+}
+
+constexpr int kLookback = 4;                // predecessors asked for per trip to memory (16 and 32: 0.5 % and 1 % slower on the 64-slice case)
+
+__device__ __forceinline__ unsigned lookback_walk(volatile unsigned* desc, int tile, int d, unsigned cnt, WsHeader* hdr) {
+    if (tile == 0) return 0;
+    unsigned excl = 0;
+    bool ok = true, done = false;
+    for (int t = tile - 1; t >= 0 && ok && !done; t -= kLookback) {
+        unsigned v[kLookback];
+#pragma unroll
+        for (int q = 0; q < kLookback; ++q) v[q] = t - q >= 0 ? desc[(size_t)(t - q) * 256 + d] : 0x80000000u;   // past tile 0: an empty prefix
+#pragma unroll
+        for (int q = 0; q < kLookback; ++q) {
+            if (done || !ok) break;
+            unsigned w = v[q];
+            int spins = 0;
+            while ((w & kFlagMask) == 0) {
+                if (++spins > kSpinLimit) { ok = false; break; }
+                __nanosleep(20);
+                w = desc[(size_t)(t - q) * 256 + d];
+            }
+            if (!ok) break;
+            excl += w & kValueMask;
+            if ((w & kFlagMask) == kFlagPrefix) done = true;
+        }
+    }
+    if (!ok) { raise_status(hdr, DST_ERR_TIMEOUT); excl = 0; }
+    desc[(size_t)tile * 256 + d] = kFlagPrefix | ((excl + cnt) & kValueMask);
+    return excl;
+}
+
+// One pass: rank the tile's keys by digit (stable), publish the tile's digit counts, lay the tile out in
+// shared memory in its sorted order while the predecessors publish theirs, fetch the cross-tile prefix,
+// then write the tile out.  Entries of one digit are consecutive in shared memory and go to consecutive
+// places in global memory, so the stores of a warp fall into a few runs instead of 32 separate sectors
+// (written straight from the registers, the scatter alone took a quarter of the pass).
+__global__ void __launch_bounds__(kRadixThreads, 2)
+k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, const unsigned* __restrict__ in_pos,
+             unsigned* __restrict__ out_keys, unsigned* __restrict__ out_pos,
+             const unsigned* __restrict__ digit_hist, unsigned* desc, int pass, int capacity,
+             const __grid_constant__ ScanArgs scan, int scan_tiles) {
+    constexpr int kWarps = kRadixThreads / 32;
+    __shared__ unsigned short wh[kWarps][256];   // counts of one tile: at most kTile, which fits 16 bits
+    __shared__ unsigned skey[kTile], spos[kTile];
+    __shared__ unsigned tile_off[256];      // where digit d starts inside the sorted tile
+    __shared__ unsigned delta[256];         // global place of entry j of digit d = delta[d] + j
+    __shared__ unsigned wsum[8], wsum2[8];
+    __shared__ unsigned s_tile;
+    pdl_trigger();
+    pdl_wait();
+    // The first CTAs of the launch are scan tiles when the row counts are known already: they need nothing
+    // from the sort, and the row-reduction kernel needs their tables only after the last pass.
+    if ((int)blockIdx.x < scan_tiles) { scan_tile(scan); return; }
+    if (threadIdx.x == 0) s_tile = atomicAdd(&hdr->ticket[pass], 1u);   // tiles start in id order
+    // asked for now, needed later: these two trips to memory overlap the ticket's
+    const unsigned n_bad = pass == 0 ? 0u : (unsigned)hdr->n_bad;
+    const bool digit_thread = threadIdx.x < 256;   // thread d < 256 looks after digit d
+    const unsigned g = digit_thread ? digit_hist[threadIdx.x] : 0u;
+    for (int s = threadIdx.x; s < kWarps * 128; s += kRadixThreads) reinterpret_cast<unsigned*>(&wh[0][0])[s] = 0;
+    __syncthreads();
+    const int tile = (int)s_tile;
+    // pass 0 reads every input position (invalid rows carry kInvalidKey and drop out);
+    // later passes read the survivors
+    const int n_in = capacity - (int)n_bad;
+    const long long t0 = (long long)tile * kTile;
+    if (t0 >= n_in) return;
+
+    const int lane = lane_id(), warp = warp_id();
+    const int shift = 8 * pass;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    unsigned key[kRadixItems], pos[kRadixItems], rank[kRadixItems];
+#pragma unroll
+    for (int k = 0; k < kRadixItems; ++k) {
+        long long e = t0 + warp * (32 * kRadixItems) + k * 32 + lane;
+        key[k] = kInvalidKey; pos[k] = 0;
+        if (e < n_in) {
+            key[k] = in_keys[e];
+            pos[k] = in_pos ? in_pos[e] : (unsigned)e;
+        }
+    }
+    // stable rank inside the warp's consecutive keys
+#pragma unroll
+    for (int k = 0; k < kRadixItems; ++k) {
+        const bool valid = key[k] != kInvalidKey;
+        unsigned dg = (key[k] >> shift) & 255u;
+        unsigned m = match_digit(dg, valid);
+        int leader = valid ? __ffs(m) - 1 : lane;
+        unsigned pre = 0;
+        if (valid && lane == leader) { pre = wh[warp][dg]; wh[warp][dg] = (unsigned short)(pre + __popc(m)); }
+        pre = __shfl_sync(0xFFFFFFFFu, pre, leader);
+        rank[k] = pre + __popc(m & lt_mask);
+        __syncwarp();
+    }
+    __syncthreads();
+    // per digit: exclusive prefix over the warps of this tile, tile total
+    const int d = threadIdx.x & 255;
+    unsigned cnt = 0;
+    if (digit_thread) {
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) { unsigned t = wh[w][d]; wh[w][d] = (unsigned short)cnt; cnt += t; }
+        lookback_publish(desc, tile, d, cnt);
+    }
+    // where digit d starts globally (exclusive scan of this pass's digit histogram) and inside the tile
+    unsigned ginc = g, tinc = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        unsigned t = __shfl_up_sync(0xFFFFFFFFu, ginc, o), u = __shfl_up_sync(0xFFFFFFFFu, tinc, o);
+        if (lane >= o) { ginc += t; tinc += u; }
+    }
+    if (lane == 31 && digit_thread) { wsum[warp] = ginc; wsum2[warp] = tinc; }
+    __syncthreads();
+    unsigned gbase = ginc - g, tbase = tinc - cnt, n_tile = 0;
+    for (int w = 0; w < 8; ++w) {
+        if (w < warp) { gbase += wsum[w]; tbase += wsum2[w]; }
+        n_tile += wsum2[w];
+    }
+    if (digit_thread) tile_off[d] = tbase;
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < kRadixItems; ++k) {
+        if (key[k] != kInvalidKey) {
+            const unsigned dg = (key[k] >> shift) & 255u;
+            const unsigned li = tile_off[dg] + wh[warp][dg] + rank[k];
+            skey[li] = key[k];
+            spos[li] = pos[k];
+        }
+    }
+    if (digit_thread) {
+        const unsigned excl = lookback_walk(desc, tile, d, cnt, hdr);
+        delta[d] = gbase + excl - tbase;
+    }
+    __syncthreads();
+    for (unsigned j = threadIdx.x; j < n_tile; j += kRadixThreads) {
+        const unsigned kk = skey[j];
+        const unsigned q = delta[(kk >> shift) & 255u] + j;
+        if (q < (unsigned)capacity) {
+            if (out_keys) out_keys[q] = kk;
+            out_pos[q] = spos[j];
+        } else {
+            raise_status(hdr, DST_ERR_TIMEOUT);   // only reachable after a failed look-back
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// a2: run lengths of the sorted keys.  The first entry of a run subtracts its position from
+// count[key], the last one adds its position + 1: two atomics per distinct row, never contended.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_bounds(const WsHeader* __restrict__ hdr, const unsigned* __restrict__ keys, unsigned* __restrict__ count,
+         int capacity, int vocab) {
+    pdl_trigger();
+    pdl_wait();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= capacity) return;
+    // the three keys and the number of valid entries are asked for together: one trip to memory.
+    // (Entries past the valid ones hold whatever the buffer held; they are read, never used.)
+    const unsigned k = keys[i];
+    const unsigned before = i > 0 ? keys[i - 1] : 0u;
+    const unsigned after = i + 1 < capacity ? keys[i + 1] : 0u;
+    const int n = capacity - (int)hdr->n_bad;
+    if (i >= n) return;
+    if (k >= (unsigned)vocab) return;                    // only after a failed look-back
+    const unsigned prev = i > 0 ? before : ~k;
+    const unsigned next = i + 1 < n ? after : ~k;
+    if (prev != k) atomicSub(&count[k], (unsigned)i);
+    if (next != k) atomicAdd(&count[k], (unsigned)i + 1u);
+}
+
 // ---- host-side launchers ------------------------------------------------------
 cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeader* hdr, unsigned* digit_hist,
-                        unsigned* keys, SliceEntry* tab, long long vocab, int passes, cudaStream_t stream) {
+                        unsigned* keys, SliceEntry* tab, long long vocab, int passes, unsigned* count, cudaStream_t stream) {
     dim3 grid(grid_x, P.n);
-    if (index_type == DST_I64)
-        return launch_pdl(k_prep<long long>, grid, dim3(kSortThreads), 0, stream, P, hdr, digit_hist, keys, tab, vocab, passes);
-    else
-        return launch_pdl(k_prep<int>, grid, dim3(kSortThreads), 0, stream, P, hdr, digit_hist, keys, tab, vocab, passes);
+    const bool wide = index_type == DST_I64;
+    if (!count) {
+        if (wide)
+            return launch_pdl(k_prep<long long, false>, grid, dim3(kPrepThreads), 0, stream, P, hdr, digit_hist, keys, tab,
+                              vocab, passes, count, 0);
+        return launch_pdl(k_prep<int, false>, grid, dim3(kPrepThreads), 0, stream, P, hdr, digit_hist, keys, tab, vocab,
+                          passes, count, 0);
+    }
+    const int words = int(((vocab + 1) / 2 + 3) / 4 * 4);
+    const size_t smem = size_t(words) * 4;
+    static SmemOptIn optin_wide, optin_narrow;
+    cudaError_t e = wide ? ensure_dynamic_smem(k_prep<long long, true>, smem, optin_wide)
+                         : ensure_dynamic_smem(k_prep<int, true>, smem, optin_narrow);
+    if (e != cudaSuccess) return e;
+    if (wide)
+        return launch_pdl(k_prep<long long, true>, grid, dim3(kPrepThreads), smem, stream, P, hdr, digit_hist, keys, tab,
+                          vocab, passes, count, words);
+    return launch_pdl(k_prep<int, true>, grid, dim3(kPrepThreads), smem, stream, P, hdr, digit_hist, keys, tab, vocab,
+                      passes, count, words);
+}
+
+static ScanArgs scan_args(const ScanParams& p) {
+    const int n_tiles = (p.vocab_pad + kScanTile - 1) / kScanTile;
+    return ScanArgs{p.hdr, p.count, p.offsets, p.heavy, p.unique_rows, p.counts_out, p.result, p.batches,
+                    p.scan_desc, p.vocab, p.vocab_pad, p.chunk, p.batch_units, n_tiles, p.wide};
 }
 
 cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
                               unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
-                              int pass, int capacity, cudaStream_t stream) {
-    return launch_pdl(k_radix_pass, dim3(n_tiles), dim3(kSortThreads), 0, stream, hdr, in_keys, in_pos, out_keys, out_pos,
-                      digit_hist, desc, pass, capacity);
+                              int pass, int capacity, const ScanParams* scan, cudaStream_t stream) {
+    ScanArgs sa{};
+    int scan_tiles = 0;
+    if (scan) { sa = scan_args(*scan); scan_tiles = sa.n_tiles; }
+    return launch_pdl(k_radix_pass, dim3(n_tiles + scan_tiles), dim3(kRadixThreads), 0, stream, hdr, in_keys, in_pos,
+                      out_keys, out_pos, digit_hist, desc, pass, capacity, sa, scan_tiles);
 }
 
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
@@ -457,12 +554,9 @@ cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* c
     return launch_pdl(k_bounds, dim3((capacity + 255) / 256), dim3(256), 0, stream, hdr, keys, count, capacity, vocab);
 }
 
-cudaError_t launch_scan(int index_type, const ScanParams& p, cudaStream_t stream) {
-    const int n_tiles = (p.vocab_pad + kScanTile - 1) / kScanTile;
-    ScanArgs s{p.hdr, p.count, p.offsets, p.heavy, p.unique_rows, p.counts_out, p.result, p.batches,
-               p.scan_desc, p.vocab, p.vocab_pad, p.chunk, p.batch_units, n_tiles};
-    if (index_type == DST_I64) return launch_pdl(k_scan<long long>, dim3(n_tiles), dim3(kScanThreads), 0, stream, s);
-    return launch_pdl(k_scan<int>, dim3(n_tiles), dim3(kScanThreads), 0, stream, s);
+cudaError_t launch_scan(const ScanParams& p, cudaStream_t stream) {
+    const ScanArgs s = scan_args(p);
+    return launch_pdl(k_scan, dim3(s.n_tiles), dim3(kScanThreads), 0, stream, s);
 }
 
 }  // namespace dst
