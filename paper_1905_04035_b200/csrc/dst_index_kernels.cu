@@ -84,14 +84,12 @@ k_prep(const __grid_constant__ HistParams P, WsHeader* __restrict__ hdr, unsigne
         if (c) atomicAdd(&digit_hist[s], c);
     }
     if (COUNT) {
-        for (int s = threadIdx.x * 4; s < count_words; s += kPrepThreads * 4) {
-            const uint4 w = *reinterpret_cast<const uint4*>(rows16 + s);
-            const unsigned ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                if (ww[q] & 0xFFFFu) atomicAdd(&count[2 * (s + q)], ww[q] & 0xFFFFu);
-                if (ww[q] >> 16) atomicAdd(&count[2 * (s + q) + 1], ww[q] >> 16);
-            }
+        // Two neighbouring rows per 64-bit add (a row's count stays below 2^32, so nothing carries over), and
+        // neighbouring lanes on neighbouring words: the adds of one instruction fall into few 32-byte sectors.
+        unsigned long long* count2 = reinterpret_cast<unsigned long long*>(count);
+        for (int s = threadIdx.x; s < count_words; s += kPrepThreads) {
+            const unsigned w = rows16[s];
+            if (w) atomicAdd(&count2[s], (unsigned long long)(w & 0xFFFFu) | ((unsigned long long)(w >> 16) << 32));
         }
     }
     for (int o = 16; o > 0; o >>= 1) bad += __shfl_down_sync(0xFFFFFFFFu, bad, o);
