@@ -177,10 +177,11 @@ static int densify_impl(const dst_slice_t* slices, int32_t R, int64_t d, int64_t
         }
         if (n_total > 0) {
             // a4: least significant digit first; keys/positions ping-pong between two buffers
+            const int items = radix_items(n_total, early_count ? scan_tile_count(int(L.vocab_pad)) : 0, sm_count());
             for (int p = 0; p < L.passes; ++p) {
                 // (the sorted keys of the last pass are read by the run-length kernel only)
                 unsigned* keys_out = early_count && p == L.passes - 1 ? nullptr : keys[(p + 1) & 1];
-                if (launch_radix_pass(int(L.n_tiles), hdr, keys[p & 1], p == 0 ? nullptr : pos[p & 1], keys_out,
+                if (launch_radix_pass(items, sm_count(), hdr, keys[p & 1], p == 0 ? nullptr : pos[p & 1], keys_out,
                                       pos[(p + 1) & 1], digit + p * 256, desc + size_t(p) * size_t(L.n_tiles) * 256, p,
                                       int(n_total), early_count && p == 0 ? &sp : nullptr, stream) != cudaSuccess)
                     return DST_ERR_CUDA;

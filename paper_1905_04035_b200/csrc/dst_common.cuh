@@ -14,8 +14,7 @@ namespace dst {
 
 // ---- fixed shape parameters -------------------------------------------------
 constexpr int kRadixThreads = 512;          // threads of a radix-pass CTA (a multiple of 256, the number of digits; 256 threads: 1 % slower on the 64-slice case)
-constexpr int kRadixItems = 8;              // keys per thread of a radix pass
-constexpr int kTile = kRadixThreads * kRadixItems;  // 4096 keys per CTA
+constexpr int kTile = kRadixThreads * 8;     // keys per CTA of a radix pass, at least (sizes the look-back descriptors)
 constexpr int kClusterCtas = 8;             // the one-kernel index path for small inputs: CTAs per cluster,
 constexpr int kFrontThreads = 1024;         // threads per CTA,
 constexpr int kFrontMaxRows = 65535;        // largest input (positions are packed into 16 bits)
@@ -252,7 +251,10 @@ struct ScanParams {
 cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeader* hdr, unsigned* digit_hist,
                         unsigned* keys, SliceEntry* tab, long long vocab, int passes, unsigned* count, cudaStream_t stream);
 // out_keys == nullptr: the last pass, whose keys nobody reads; scan != nullptr: the scan tiles ride in this launch
-cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
+// items: keys per thread, from radix_items(); a pass over n keys then has ceil(n / (kRadixThreads * items)) tiles
+int radix_items(long long n, int extra_ctas, int sms);
+int scan_tile_count(int vocab_pad);
+cudaError_t launch_radix_pass(int items, int sms, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
                               unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
                               int pass, int capacity, const ScanParams* scan, cudaStream_t stream);
 struct FrontParams {

@@ -373,14 +373,23 @@ __device__ __forceinline__ unsigned lookback_walk(volatile unsigned* desc, int t
 // then write the tile out.  Entries of one digit are consecutive in shared memory and go to consecutive
 // places in global memory, so the stores of a warp fall into a few runs instead of 32 separate sectors
 // (written straight from the registers, the scatter alone took a quarter of the pass).
-__global__ void __launch_bounds__(kRadixThreads, 2)
+//
+// ITEMS keys per thread, kRadixThreads * ITEMS per tile: the host picks the smallest tile with which every CTA of
+// the launch has an SM of its own (two CTAs on one SM rank their keys at half the speed, and every tile after
+// them in the order waits for their counts).  With all CTAs resident from the start the tile number is the CTA
+// number; otherwise tiles take a ticket, so that a tile's predecessors are running or done when it starts.
+template <int ITEMS>
+__global__ void __launch_bounds__(kRadixThreads, ITEMS <= 8 ? 2 : 1)
 k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, const unsigned* __restrict__ in_pos,
              unsigned* __restrict__ out_keys, unsigned* __restrict__ out_pos,
              const unsigned* __restrict__ digit_hist, unsigned* desc, int pass, int capacity,
-             const __grid_constant__ ScanArgs scan, int scan_tiles) {
+             const __grid_constant__ ScanArgs scan, int scan_tiles, int ticketed) {
     constexpr int kWarps = kRadixThreads / 32;
-    __shared__ unsigned short wh[kWarps][256];   // counts of one tile: at most kTile, which fits 16 bits
-    __shared__ unsigned skey[kTile], spos[kTile];
+    constexpr int kTileKeys = kRadixThreads * ITEMS;
+    __shared__ unsigned short wh[kWarps][256];   // counts of one tile: at most 8192, which fits 16 bits
+    extern __shared__ __align__(16) unsigned staged[];
+    unsigned* skey = staged;
+    unsigned* spos = staged + kTileKeys;
     __shared__ unsigned tile_off[256];      // where digit d starts inside the sorted tile
     __shared__ unsigned delta[256];         // global place of entry j of digit d = delta[d] + j
     __shared__ unsigned wsum[8], wsum2[8];
@@ -390,7 +399,7 @@ k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, c
     // The first CTAs of the launch are scan tiles when the row counts are known already: they need nothing
     // from the sort, and the row-reduction kernel needs their tables only after the last pass.
     if ((int)blockIdx.x < scan_tiles) { scan_tile(scan); return; }
-    if (threadIdx.x == 0) s_tile = atomicAdd(&hdr->ticket[pass], 1u);   // tiles start in id order
+    if (threadIdx.x == 0) s_tile = ticketed ? atomicAdd(&hdr->ticket[pass], 1u) : blockIdx.x - (unsigned)scan_tiles;
     // asked for now, needed later: these two trips to memory overlap the ticket's
     const unsigned n_bad = pass == 0 ? 0u : (unsigned)hdr->n_bad;
     const bool digit_thread = threadIdx.x < 256;   // thread d < 256 looks after digit d
@@ -401,16 +410,16 @@ k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, c
     // pass 0 reads every input position (invalid rows carry kInvalidKey and drop out);
     // later passes read the survivors
     const int n_in = capacity - (int)n_bad;
-    const long long t0 = (long long)tile * kTile;
+    const long long t0 = (long long)tile * kTileKeys;
     if (t0 >= n_in) return;
 
     const int lane = lane_id(), warp = warp_id();
     const int shift = 8 * pass;
     const unsigned lt_mask = (1u << lane) - 1u;
-    unsigned key[kRadixItems], pos[kRadixItems], rank[kRadixItems];
+    unsigned key[ITEMS], pos[ITEMS], rank[ITEMS];
 #pragma unroll
-    for (int k = 0; k < kRadixItems; ++k) {
-        long long e = t0 + warp * (32 * kRadixItems) + k * 32 + lane;
+    for (int k = 0; k < ITEMS; ++k) {
+        long long e = t0 + warp * (32 * ITEMS) + k * 32 + lane;
         key[k] = kInvalidKey; pos[k] = 0;
         if (e < n_in) {
             key[k] = in_keys[e];
@@ -419,7 +428,7 @@ k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, c
     }
     // stable rank inside the warp's consecutive keys
 #pragma unroll
-    for (int k = 0; k < kRadixItems; ++k) {
+    for (int k = 0; k < ITEMS; ++k) {
         const bool valid = key[k] != kInvalidKey;
         unsigned dg = (key[k] >> shift) & 255u;
         unsigned m = match_digit(dg, valid);
@@ -456,7 +465,7 @@ k_radix_pass(WsHeader* __restrict__ hdr, const unsigned* __restrict__ in_keys, c
     if (digit_thread) tile_off[d] = tbase;
     __syncthreads();
 #pragma unroll
-    for (int k = 0; k < kRadixItems; ++k) {
+    for (int k = 0; k < ITEMS; ++k) {
         if (key[k] != kInvalidKey) {
             const unsigned dg = (key[k] >> shift) & 255u;
             const unsigned li = tile_off[dg] + wh[warp][dg] + rank[k];
@@ -531,20 +540,56 @@ cudaError_t launch_prep(const HistParams& P, int grid_x, int index_type, WsHeade
                       passes, count, words);
 }
 
+int scan_tile_count(int vocab_pad) { return (vocab_pad + kScanTile - 1) / kScanTile; }
+
 static ScanArgs scan_args(const ScanParams& p) {
-    const int n_tiles = (p.vocab_pad + kScanTile - 1) / kScanTile;
+    const int n_tiles = scan_tile_count(p.vocab_pad);
     return ScanArgs{p.hdr, p.count, p.offsets, p.heavy, p.unique_rows, p.counts_out, p.result, p.batches,
                     p.scan_desc, p.vocab, p.vocab_pad, p.chunk, p.batch_units, n_tiles, p.wide};
 }
 
-cudaError_t launch_radix_pass(int n_tiles, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
+// Items per thread of a radix pass over n keys, given the CTAs that ride along and the SMs of the device.
+int radix_items(long long n, int extra_ctas, int sms) {
+    const int choices[4] = {8, 10, 12, 16};
+    for (int c = 0; c < 4; ++c) {
+        const long long tile = (long long)kRadixThreads * choices[c];
+        if ((n + tile - 1) / tile + extra_ctas <= sms) return choices[c];
+    }
+    return n > 4LL * sms * kRadixThreads * 8 ? 16 : 8;
+}
+
+template <int ITEMS>
+static cudaError_t launch_radix_as(int n_tiles, cudaStream_t stream, int sms, WsHeader* hdr, const unsigned* in_keys,
+                                   const unsigned* in_pos, unsigned* out_keys, unsigned* out_pos,
+                                   const unsigned* digit_hist, unsigned* desc, int pass, int capacity,
+                                   const ScanArgs& sa, int scan_tiles) {
+    static SmemOptIn optin;
+    const size_t smem = size_t(kRadixThreads) * ITEMS * 8;
+    cudaError_t e = ensure_dynamic_smem(k_radix_pass<ITEMS>, smem, optin);
+    if (e != cudaSuccess) return e;
+    const int ticketed = n_tiles + scan_tiles > sms ? 1 : 0;
+    return launch_pdl(k_radix_pass<ITEMS>, dim3(n_tiles + scan_tiles), dim3(kRadixThreads), smem, stream, hdr, in_keys,
+                      in_pos, out_keys, out_pos, digit_hist, desc, pass, capacity, sa, scan_tiles, ticketed);
+}
+
+cudaError_t launch_radix_pass(int items, int sms, WsHeader* hdr, const unsigned* in_keys, const unsigned* in_pos,
                               unsigned* out_keys, unsigned* out_pos, const unsigned* digit_hist, unsigned* desc,
                               int pass, int capacity, const ScanParams* scan, cudaStream_t stream) {
     ScanArgs sa{};
     int scan_tiles = 0;
     if (scan) { sa = scan_args(*scan); scan_tiles = sa.n_tiles; }
-    return launch_pdl(k_radix_pass, dim3(n_tiles + scan_tiles), dim3(kRadixThreads), 0, stream, hdr, in_keys, in_pos,
-                      out_keys, out_pos, digit_hist, desc, pass, capacity, sa, scan_tiles);
+    const int tile = kRadixThreads * items;
+    const int n_tiles = (capacity + tile - 1) / tile;
+#define DST_RADIX_CASE(I) case I: return launch_radix_as<I>(n_tiles, stream, sms, hdr, in_keys, in_pos, out_keys, out_pos, \
+                                                            digit_hist, desc, pass, capacity, sa, scan_tiles)
+    switch (items) {
+        DST_RADIX_CASE(8);
+        DST_RADIX_CASE(10);
+        DST_RADIX_CASE(12);
+        DST_RADIX_CASE(16);
+    }
+#undef DST_RADIX_CASE
+    return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_bounds(const WsHeader* hdr, const unsigned* keys, unsigned* count, int capacity, int vocab,
