@@ -34,7 +34,7 @@ constexpr int kPipeHeaderReserve = 1024;    // mbarriers in front of the slots
 constexpr int kMaxBlockCols = 1024;         // columns per column block (32 fp32 accumulators per lane)
 constexpr long long kWaitCycles = 1LL << 31; // SM clock cycles (about a second) before an mbarrier wait gives up
 constexpr int kScanThreads = kRadixThreads;  // the scan tiles can ride in the launch of the first radix pass
-constexpr int kScanItems = 4;               // rows per thread in the scan kernel (16: 2 % slower on r64, 8: 0.5 %)
+constexpr int kScanItems = 4;               // rows per thread of a scan tile (8: the scan tiles outlast the first radix pass they ride in)
 constexpr int kScanTile = kScanThreads * kScanItems;
 constexpr int kSmCount = 148;               // B200; only used to pick the chunk length
 constexpr unsigned kInvalidKey = 0xFFFFFFFFu;
@@ -193,6 +193,15 @@ inline Layout make_layout(int64_t n_rows, int32_t R, int64_t d, int64_t vocab, i
         int pow2 = 8;                                     // the small-input path cuts items of the power of two below batch_units
         while (pow2 * 2 <= L.batch_units) pow2 *= 2;
         L.batch_max = (vocab + n_rows) / pow2 + 2;
+    }
+    // A large input that names one row only is nothing but chunk items of equal length: cut them so that a whole
+    // number of rounds gives every warp the same number (with 128 entries, 3.46 items per warp meant four rounds
+    // for some warps and three for others).  Small inputs keep the power of two their index path needs.
+    if (c == max_chunk && n_rows > kFrontMaxRows) {
+        const int64_t warps = int64_t(kSmCount) * (value_size == 2 ? 16 : 8);
+        const int64_t rounds = (n_rows + warps * max_chunk - 1) / (warps * max_chunk);
+        const int64_t even = (n_rows + warps * rounds - 1) / (warps * rounds);
+        if (even >= max_chunk / 2 && even <= max_chunk) c = int(even);
     }
     L.chunk = c;
     int bits = 0;
