@@ -39,18 +39,21 @@ ALL_CONFIGS = ("tiny", "base", "big", "r64", "sweep_uniform", "sweep_zipf", "swe
 # the two workloads with a stated bar: at least this fraction of the measured HBM peak for the whole step
 TARGETS = {"big": 0.70, "r64": 0.70}
 TRAFFIC_FILE = os.path.join(ROOT, "profiles", "k_reduce_rows_dram_traffic.txt")
-KERNEL_SOURCE = os.path.join(ROOT, "paper_1905_04035_b200", "csrc", "dst_reduce_kernels.cu")
+KERNEL_SOURCES = [os.path.join(ROOT, "paper_1905_04035_b200", "csrc", f) for f in ("dst_reduce_kernels.cu", "dst_common.cuh")]
 
 
 def kernel_dram_traffic(workload: str):
     """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the row-reduction kernel on `workload`, as an ncu
-    capture recorded it in profiles/k_reduce_rows_dram_traffic.txt (lines: workload, bytes, sha256 of the kernel's
-    source file at capture time).  None when there is no record for the workload, or when the kernel's source
-    has changed since: counters of another kernel are not this kernel's traffic."""
+    capture recorded it in profiles/k_reduce_rows_dram_traffic.txt (lines: workload, bytes, sha256 over the kernel's
+    source file and the header it shares with the other kernels, at capture time).  None when there is no record for
+    the workload, or when the sources have changed since: counters of another kernel are not this kernel's traffic."""
     import hashlib
     try:
-        with open(KERNEL_SOURCE, "rb") as f:
-            now = hashlib.sha256(f.read()).hexdigest()
+        h = hashlib.sha256()
+        for path in KERNEL_SOURCES:
+            with open(path, "rb") as f:
+                h.update(f.read())
+        now = h.hexdigest()
         for line in open(TRAFFIC_FILE):
             f = line.split()
             if len(f) >= 3 and not line.startswith("#") and f[0] == workload:
