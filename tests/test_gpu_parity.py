@@ -161,6 +161,27 @@ def test_radix_pass_counts(vocab, passes):
     assert_parity(w, run_library(w))
 
 
+@pytest.mark.parametrize("vocab,ns", [
+    (33707, [9000] * 70),                     # odd vocabulary; more slices than one validation launch describes
+    (65536, [20000, 0, 8192, 8193, 40000]),   # largest vocabulary counted in shared memory; slices of several CTAs
+    (65537, [70000]),                         # one more row: counts come from the sorted keys instead
+    (513, [100000]),                          # every row heavy; two digits, the second nearly empty
+])
+def test_row_counts_taken_while_validating(vocab, ns):
+    """Large inputs over a small vocabulary: the validation kernel counts the rows and the scan rides in the first
+    radix pass.  Runs of one row longer than a warp (the one-add-per-warp case), with out-of-range and negative
+    indices inside them, and rows at both ends of the vocabulary."""
+    def idx(rng, k):
+        ix = rng.integers(0, vocab, size=k)
+        run = np.arange(k) % 1000 < 200            # 200 consecutive entries of one row in every 1000
+        ix[run] = (np.arange(k)[run] // 1000) % 2 * (vocab - 1)
+        ix[5::997] = vocab + 3
+        ix[6::1499] = -1
+        return ix
+    w = _custom(vocab, 64, ns, idx_fn=idx, integer=True)
+    assert_parity(w, run_library(w))
+
+
 @pytest.mark.parametrize("d", [8, 64, 136, 520, 1024, 2056, 4096])
 def test_row_widths(d):
     w = _custom(300, d, [2500], idx_fn=lambda rng, n: np.minimum(rng.zipf(1.3, size=n) - 1, 299))
