@@ -595,15 +595,22 @@ struct WarpPipe {
             issued_mask &= ~(1u << cslot);
             const char* sp = ring_ptr + (size_t)cslot * a.slot_bytes;
             if (kind & kUnitAdd) {
-                Acc<VC> v[K];
+                // A block of full width (the usual case) takes plain loads: one predicate and eight cleared registers
+                // per column group, in every unit, were a tenth of the bf16 kernel's instructions.  Only here, where
+                // most units pass: the same split at the closing units made the short optimizer kernels slower.
+                if (wcols == K * 32 * VC) {
+                    Acc<VC> v[K];
 #pragma unroll
-                for (int k = 0; k < K; ++k) {
-                    const int c = col(k);
-                    zero(v[k]);
-                    if (c < wcols) load_elems(reinterpret_cast<const VT*>(sp) + c, v[k]);
+                    for (int k = 0; k < K; ++k) load_elems(reinterpret_cast<const VT*>(sp) + col(k), v[k]);
+#pragma unroll
+                    for (int k = 0; k < K; ++k) add(acc[k], v[k]);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        const int c = col(k);
+                        if (c < wcols) { Acc<VC> v; load_elems(reinterpret_cast<const VT*>(sp) + c, v); add(acc[k], v); }
+                    }
                 }
-#pragma unroll
-                for (int k = 0; k < K; ++k) add(acc[k], v[k]);
             }
             if (kind & kUnitAddDense) {
                 Acc<VC> v[K];
