@@ -597,8 +597,9 @@ struct WarpPipe {
             if (kind & kUnitAdd) {
                 // A block of full width (the usual case) takes plain loads: one predicate and eight cleared registers
                 // per column group, in every unit, were a tenth of the bf16 kernel's instructions.  Only here, where
-                // most units pass: the same split at the closing units made the short optimizer kernels slower.
-                if (wcols == K * 32 * VC) {
+                // most units pass, and not in the optimizer kernels: the same split at the closing units, or in the
+                // Adam kernel (200 registers as it is), made those slower.
+                if (OPT == kOptNone && wcols == K * 32 * VC) {
                     Acc<VC> v[K];
 #pragma unroll
                     for (int k = 0; k < K; ++k) load_elems(reinterpret_cast<const VT*>(sp) + col(k), v[k]);
