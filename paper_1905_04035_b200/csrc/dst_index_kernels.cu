@@ -7,10 +7,12 @@
 // plus the work-item tables the row-reduction kernel consumes.  Integer work only.
 //
 // Order of the kernels (large inputs):
-//   k_prep        validate, narrow to 32-bit keys, digit histograms of all radix passes
-//   k_radix_pass  one per 8-bit digit, least significant first, stable
-//   k_bounds      run lengths of the sorted keys -> count[v]
-//   k_scan        count[] -> offsets, unique rows, heavy-row chunks, row batches
+//   k_prep        validate, narrow to 32-bit keys, digit histograms of all radix passes; for vocabularies of
+//                 at most 65536 rows also count[v], in shared memory
+//   k_radix_pass  one per 8-bit digit, least significant first, stable; when count[] is known already, the scan
+//                 tiles ride in the launch of the first pass and nothing else follows the last one
+//   k_bounds      (larger vocabularies) run lengths of the sorted keys -> count[v]
+//   k_scan        (larger vocabularies) count[] -> offsets, unique rows, heavy-row chunks, row batches
 // Small inputs take k_front_cluster (dst_front_cluster.cu), which does all of it in one kernel.
 #include "dst_common.cuh"
 
