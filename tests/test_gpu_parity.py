@@ -7,7 +7,7 @@ import oracle
 import paper_1905_04035_b200 as dst
 from paper_1905_04035_b200.workloads import Workload, make_workload, to_bf16_bits
 
-from gpu_helpers import assert_parity, oracle_of, raw_bits, run_library, to_device, to_numpy_f64
+from gpu_helpers import TORCH_DT, assert_parity, oracle_of, raw_bits, run_library, to_device, to_numpy_f64, tolerance
 
 pytestmark = pytest.mark.gpu
 
@@ -425,3 +425,30 @@ def test_nvtx_ranges_can_be_switched_on_and_change_nothing():
     finally:
         dst.dst_profile_ranges(False)
     assert np.array_equal(raw_bits(plain.out), raw_bits(ranged.out))
+
+
+# ---------------------------------------------------------------------------
+# nothing may depend on what the workspace held before the call
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("name,scale", [("tiny", 1.0), ("base", 1.0), ("r64", 0.05), ("sweep_zipf", 0.02)])
+def test_a_dirty_workspace_changes_nothing(name, scale):
+    """The workspace is filled with 0xFF, then with 0x01 (every flag and counter of a header 'set'), and is also
+    used as an earlier call left it: all four outputs are bit-identical and within tolerance of the oracle."""
+    w = make_workload(name, scale=scale)
+    idt, vdt, odt = TORCH_DT[w.index_dtype], TORCH_DT[w.value_dtype], TORCH_DT[w.out_dtype]
+    slices = [(to_device(i, w.index_dtype), to_device(v, w.value_dtype)) for i, v in zip(w.indices, w.values)]
+    dense = to_device(w.dense_in, w.out_dtype) if w.dense_in is not None else None
+    eng = dst.Densifier(w.n_rows_total, len(slices), w.d, w.vocab, index_dtype=idt, value_dtype=vdt, out_dtype=odt)
+    outs = []
+    for fill in (0xFF, None, 0x01, None):
+        if fill is not None:
+            eng.workspace.fill_(fill)
+        out = torch.full((w.vocab, w.d), float("nan"), dtype=odt, device="cuda")
+        eng(slices, dense, out)
+        torch.cuda.synchronize()
+        assert eng.read_result()["status"] == 0
+        outs.append(out)
+    for o in outs[1:]:
+        assert np.array_equal(raw_bits(o), raw_bits(outs[0]))
+    orc = oracle_of(w)
+    assert np.all(np.abs(to_numpy_f64(outs[0]) - orc.acc) <= tolerance(w, orc))
